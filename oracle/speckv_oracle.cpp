@@ -1,0 +1,466 @@
+/*
+ * SpecKV oracle -- TEST INFRASTRUCTURE ONLY (see speckv_oracle.h).
+ *
+ * Plain C++17, double precision, sequential loops over the vocabulary; std::thread
+ * is used across batch rows only (rows are independent).  No blocking, fusion or
+ * reordering beyond what each definition states:
+ *
+ *   signals      paper Sec. 4.2: H(q_i) = -sum_v q_i(v) log q_i(v), c_i = max_v q_i(v),
+ *                Hbar, cbar = means over the gamma drafted positions, Hmax, cmin.
+ *   controller   paper Sec. 4.3: context vector -> 16 hidden units -> one predicted
+ *                acceptance rate per candidate gamma; Eq. 1: E = a_hat * gamma + 1;
+ *                gamma* = argmax.
+ *   verification paper Sec. 3.1 (greedy: accept while the target's top prediction equals
+ *                the draft token; the target's prediction replaces the first mismatch; a
+ *                bonus prediction follows a fully accepted draft; tokens per step = k + 1),
+ *                and, for temperature > 0, the lossless speculative-sampling rule the
+ *                paper cites (Sec. 1, 2.1): accept x_i while u_i < min(1, p(x_i)/q(x_i));
+ *                the first rejected position is resampled from norm(max(0, p - q)); a
+ *                fully accepted draft gets a bonus token from p.
+ *
+ * Readings fixed where the paper is silent (the same list is kept in the design notes):
+ *   - entropy in nats by default, bits on request (the paper writes log2);
+ *   - signals use the draft softmax at the row's temperature; greedy rows (T = 0) use T = 1;
+ *   - accept test evaluated as ln u + ln q(x) < ln p(x); q(x) = 0 accepts iff p(x) > 0;
+ *   - uniforms are indexed by position: u[b,i,0] accept test, u[b,n,1] resample / bonus;
+ *   - inverse CDF in vocabulary order: smallest v with cumulative weight > u * total,
+ *     falling back to the last v with positive weight;
+ *   - argmax ties go to the lowest index (token id, and candidate gamma);
+ *   - -inf logits are legal (probability 0); NaN, +inf or an all -inf row flag the row.
+ */
+#include "speckv_oracle.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <limits>
+#include <thread>
+#include <vector>
+
+namespace {
+
+inline double load_logit(const void* base, int32_t dtype, int64_t idx) {
+    if (dtype == ORACLE_DT_F32) {
+        return static_cast<double>(static_cast<const float*>(base)[idx]);
+    }
+    uint16_t h = static_cast<const uint16_t*>(base)[idx];
+    uint32_t w = static_cast<uint32_t>(h) << 16;
+    float f;
+    std::memcpy(&f, &w, sizeof f);
+    return static_cast<double>(f);
+}
+
+struct RowRef {
+    const void* base;
+    int32_t dtype;
+    int64_t off;
+    double at(int64_t v) const { return load_logit(base, dtype, off + v); }
+};
+
+/* max and log-sum-exp of x_v / T; returns false when the row is unusable */
+bool lse_row(const RowRef& r, int32_t V, double T, double* m_out, double* lnZ_out) {
+    double m = -std::numeric_limits<double>::infinity();
+    for (int32_t v = 0; v < V; ++v) {
+        double x = r.at(v);
+        if (std::isnan(x) || x == std::numeric_limits<double>::infinity()) return false;
+        x /= T;
+        if (x > m) m = x;
+    }
+    if (!(m > -std::numeric_limits<double>::infinity())) return false;
+    double Z = 0.0;
+    for (int32_t v = 0; v < V; ++v) Z += std::exp(r.at(v) / T - m);
+    *m_out = m;
+    *lnZ_out = std::log(Z);
+    return true;
+}
+
+bool softmax_row(const RowRef& r, int32_t V, double T, double* prob) {
+    double m = -std::numeric_limits<double>::infinity();
+    for (int32_t v = 0; v < V; ++v) {
+        double x = r.at(v);
+        if (std::isnan(x) || x == std::numeric_limits<double>::infinity()) return false;
+        x /= T;
+        if (x > m) m = x;
+    }
+    if (!(m > -std::numeric_limits<double>::infinity())) return false;
+    double Z = 0.0;
+    for (int32_t v = 0; v < V; ++v) {
+        prob[v] = std::exp(r.at(v) / T - m);
+        Z += prob[v];
+    }
+    for (int32_t v = 0; v < V; ++v) prob[v] /= Z;
+    return true;
+}
+
+double entropy_nats(const double* q, int32_t V) {
+    double H = 0.0;
+    for (int32_t v = 0; v < V; ++v)
+        if (q[v] > 0.0) H -= q[v] * std::log(q[v]);
+    return H;
+}
+
+/* lowest index of the maximum; -1 when the row holds NaN / +inf or only -inf */
+int32_t argmax_row(const RowRef& r, int32_t V) {
+    double best = -std::numeric_limits<double>::infinity();
+    int32_t arg = -1;
+    for (int32_t v = 0; v < V; ++v) {
+        double x = r.at(v);
+        if (std::isnan(x) || x == std::numeric_limits<double>::infinity()) return -1;
+        if (x > best) {
+            best = x;
+            arg = v;
+        }
+    }
+    return arg;
+}
+
+int32_t inverse_cdf(const double* w, int32_t V, double u, int32_t* near_boundary) {
+    double W = 0.0;
+    for (int32_t v = 0; v < V; ++v) W += w[v];
+    if (near_boundary) *near_boundary = 0;
+    if (!(W > 0.0)) return -1;
+    const double tau = u * W;
+    double cum = 0.0, lower = 0.0;
+    int32_t chosen = -1, last_pos = -1;
+    for (int32_t v = 0; v < V; ++v) {
+        if (w[v] > 0.0) last_pos = v;
+        double next = cum + w[v];
+        if (next > tau) {
+            chosen = v;
+            lower = cum;
+            cum = next;
+            break;
+        }
+        cum = next;
+    }
+    if (chosen < 0) {
+        chosen = last_pos;
+        if (near_boundary) *near_boundary = 1;
+        return chosen;
+    }
+    if (near_boundary) {
+        const double eps = 1e-6 * W;
+        /* upper boundary of the chosen token, and its lower boundary (= upper boundary of
+         * the previous token with positive weight); the lower one only matters if a token
+         * with positive weight precedes the chosen one */
+        bool near_hi = std::fabs(cum - tau) < eps;
+        bool near_lo = (lower > 0.0) && std::fabs(tau - lower) < eps;
+        *near_boundary = (near_hi || near_lo) ? 1 : 0;
+    }
+    return chosen;
+}
+
+struct RowParams {
+    int32_t gamma;
+    double T;      /* temperature as given (0 => greedy) */
+    int32_t status;
+};
+
+RowParams row_params(const oracle_batch* bt, int32_t b) {
+    RowParams rp;
+    rp.status = ORACLE_ROW_OK;
+    rp.gamma = bt->gamma ? bt->gamma[b] : bt->gamma_max;
+    float tf = bt->temperature ? bt->temperature[b] : bt->temperature_scalar;
+    rp.T = static_cast<double>(tf);
+    if (rp.gamma < 1 || rp.gamma > bt->gamma_max) rp.status |= ORACLE_ROW_BAD_GAMMA;
+    if (!(rp.T >= 0.0) || std::isinf(rp.T)) rp.status |= ORACLE_ROW_BAD_TEMPERATURE;
+    return rp;
+}
+
+inline RowRef draft_row(const oracle_batch* bt, int32_t b, int32_t i) {
+    return RowRef{bt->draft, bt->dtype,
+                  static_cast<int64_t>(b) * bt->draft_stride_row +
+                      static_cast<int64_t>(i) * bt->draft_stride_pos};
+}
+inline RowRef target_row(const oracle_batch* bt, int32_t b, int32_t i) {
+    return RowRef{bt->target, bt->dtype,
+                  static_cast<int64_t>(b) * bt->target_stride_row +
+                      static_cast<int64_t>(i) * bt->target_stride_pos};
+}
+
+/* ---- signals, one batch row (paper Sec. 4.2) ---- */
+void signals_row(const oracle_batch* bt, int32_t b, double* H, double* C, double* feat,
+                 int32_t* row_status) {
+    const int32_t G = bt->gamma_max, V = bt->V;
+    double* Hb = H ? H + static_cast<int64_t>(b) * G : nullptr;
+    double* Cb = C ? C + static_cast<int64_t>(b) * G : nullptr;
+    double* fb = feat ? feat + static_cast<int64_t>(b) * 4 : nullptr;
+    if (Hb) std::fill(Hb, Hb + G, 0.0);
+    if (Cb) std::fill(Cb, Cb + G, 0.0);
+    if (fb) std::fill(fb, fb + 4, 0.0);
+
+    RowParams rp = row_params(bt, b);
+    if (rp.status) {
+        if (row_status) row_status[b] |= rp.status;
+        return;
+    }
+    const double Tsig = (rp.T == 0.0) ? 1.0 : rp.T;
+    std::vector<double> q(V), Hi(rp.gamma), Ci(rp.gamma);
+    for (int32_t i = 0; i < rp.gamma; ++i) {
+        if (!softmax_row(draft_row(bt, b, i), V, Tsig, q.data())) {
+            if (row_status) row_status[b] |= ORACLE_ROW_NONFINITE;
+            return;
+        }
+        double h = entropy_nats(q.data(), V);
+        if (bt->entropy_in_bits) h /= std::log(2.0);
+        Hi[i] = h;
+        Ci[i] = *std::max_element(q.begin(), q.end());
+    }
+    double Hsum = 0.0, Csum = 0.0, Hmax = Hi[0], Cmin = Ci[0];
+    for (int32_t i = 0; i < rp.gamma; ++i) {
+        Hsum += Hi[i];
+        Csum += Ci[i];
+        Hmax = std::max(Hmax, Hi[i]);
+        Cmin = std::min(Cmin, Ci[i]);
+        if (Hb) Hb[i] = Hi[i];
+        if (Cb) Cb[i] = Ci[i];
+    }
+    if (fb) {
+        fb[0] = Hsum / rp.gamma;
+        fb[1] = Csum / rp.gamma;
+        fb[2] = Hmax;
+        fb[3] = Cmin;
+    }
+}
+
+/* ---- controller, one row (paper Sec. 4.3, Eq. 1) ---- */
+void select_gamma_row(const double* feat4, const float* comp, const oracle_mlp* mlp, double* scores,
+                      int32_t* gamma_next, int32_t* near) {
+    std::vector<double> x(mlp->n_in, 0.0);
+    if (mlp->feature_layout == 0) {
+        /* mean entropy, mean confidence, min confidence, two compression flags */
+        x[0] = feat4[0];
+        x[1] = feat4[1];
+        x[2] = feat4[3];
+        for (int32_t k = 3; k < mlp->n_in; ++k) x[k] = comp ? static_cast<double>(comp[k - 3]) : 0.0;
+    } else {
+        /* the paper's context vector [Hbar, cbar, Hmax, cmin, comp] */
+        x[0] = feat4[0];
+        x[1] = feat4[1];
+        x[2] = feat4[2];
+        x[3] = feat4[3];
+        for (int32_t k = 4; k < mlp->n_in; ++k) x[k] = comp ? static_cast<double>(comp[k - 4]) : 0.0;
+    }
+    std::vector<double> h(mlp->n_hidden);
+    for (int32_t k = 0; k < mlp->n_hidden; ++k) {
+        double a = static_cast<double>(mlp->b1[k]);
+        for (int32_t f = 0; f < mlp->n_in; ++f)
+            a += static_cast<double>(mlp->W1[static_cast<int64_t>(k) * mlp->n_in + f]) * x[f];
+        h[k] = a > 0.0 ? a : 0.0;
+    }
+    int32_t best = 0;
+    double best_e = 0.0, second_e = -std::numeric_limits<double>::infinity();
+    for (int32_t j = 0; j < mlp->n_out; ++j) {
+        double o = static_cast<double>(mlp->b2[j]);
+        for (int32_t k = 0; k < mlp->n_hidden; ++k)
+            o += static_cast<double>(mlp->W2[static_cast<int64_t>(j) * mlp->n_hidden + k]) * h[k];
+        double e = (mlp->score_transform == 0) ? o * mlp->gamma_choices[j] + 1.0 : o;
+        if (scores) scores[j] = e;
+        if (j == 0) {
+            best_e = e;
+        } else if (e > best_e) {
+            second_e = best_e;
+            best_e = e;
+            best = j;
+        } else if (e > second_e) {
+            second_e = e;
+        }
+    }
+    if (gamma_next) *gamma_next = mlp->gamma_choices[best];
+    if (near) {
+        bool tie = (mlp->n_out > 1) && (best_e - second_e) < 1e-5 * std::max(std::fabs(best_e), 1e-30);
+        if (tie) *near |= ORACLE_NEAR_GAMMA;
+    }
+}
+
+/* ---- verification, one row ---- */
+void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t* out_tokens,
+                int32_t* row_status, int32_t* near) {
+    const int32_t G = bt->gamma_max, V = bt->V;
+    int32_t* ob = out_tokens + static_cast<int64_t>(b) * (G + 1);
+    std::fill(ob, ob + G + 1, -1);
+    n_accepted[b] = 0;
+
+    RowParams rp = row_params(bt, b);
+    if (rp.status) {
+        if (row_status) row_status[b] |= rp.status;
+        return;
+    }
+    const int32_t g = rp.gamma;
+    const int32_t* xb = bt->draft_tokens + static_cast<int64_t>(b) * G;
+    int32_t st = ORACLE_ROW_OK;
+    for (int32_t i = 0; i < g; ++i)
+        if (xb[i] < 0 || xb[i] >= V) st |= ORACLE_ROW_BAD_TOKEN;
+
+    int32_t n = g, fresh = -1, nearbits = 0;
+
+    if (rp.T == 0.0) {
+        /* greedy rule of Sec. 3.1.  Every target row the step uses is checked first. */
+        std::vector<int32_t> am(g + 1);
+        for (int32_t i = 0; i <= g; ++i) {
+            am[i] = argmax_row(target_row(bt, b, i), V);
+            if (am[i] < 0) st |= ORACLE_ROW_NONFINITE;
+        }
+        for (int32_t i = 0; i < g; ++i)
+            if (argmax_row(draft_row(bt, b, i), V) < 0) st |= ORACLE_ROW_NONFINITE;
+        if (st) {
+            if (row_status) row_status[b] |= st;
+            return;
+        }
+        for (int32_t i = 0; i < g; ++i) {
+            if (xb[i] != am[i]) {
+                n = i;
+                break;
+            }
+        }
+        fresh = am[n];
+    } else {
+        const double T = rp.T;
+        std::vector<double> mq(g), lzq(g), mp(g + 1), lzp(g + 1);
+        for (int32_t i = 0; i < g; ++i)
+            if (!lse_row(draft_row(bt, b, i), V, T, &mq[i], &lzq[i])) st |= ORACLE_ROW_NONFINITE;
+        for (int32_t i = 0; i <= g; ++i)
+            if (!lse_row(target_row(bt, b, i), V, T, &mp[i], &lzp[i])) st |= ORACLE_ROW_NONFINITE;
+        if (st) {
+            if (row_status) row_status[b] |= st;
+            return;
+        }
+        const float* ub = bt->uniforms + static_cast<int64_t>(b) * (G + 1) * 2;
+        for (int32_t i = 0; i < g; ++i) {
+            const double u = static_cast<double>(ub[2 * i + 0]);
+            const double lnq = draft_row(bt, b, i).at(xb[i]) / T - mq[i] - lzq[i];
+            const double lnp = target_row(bt, b, i).at(xb[i]) / T - mp[i] - lzp[i];
+            const double ratio = std::exp(lnp - lnq); /* p(x)/q(x); inf when q(x) = 0 < p(x) */
+            if (std::fabs(u - ratio) < 1e-6) nearbits |= ORACLE_NEAR_ACCEPT;
+            /* accept iff u*q(x) < p(x) */
+            const bool accept = (std::log(u) + lnq) < lnp;
+            if (!accept) {
+                n = i;
+                break;
+            }
+        }
+        std::vector<double> p(V), w(V);
+        softmax_row(target_row(bt, b, n), V, T, p.data());
+        const double u2 = static_cast<double>(ub[2 * n + 1]);
+        int32_t nb = 0;
+        if (n < g) {
+            std::vector<double> q(V);
+            softmax_row(draft_row(bt, b, n), V, T, q.data());
+            for (int32_t v = 0; v < V; ++v) w[v] = std::max(0.0, p[v] - q[v]);
+            fresh = inverse_cdf(w.data(), V, u2, &nb);
+            if (fresh < 0) fresh = inverse_cdf(p.data(), V, u2, &nb); /* p == q numerically */
+        } else {
+            fresh = inverse_cdf(p.data(), V, u2, &nb);
+        }
+        if (nb) nearbits |= ORACLE_NEAR_CDF;
+    }
+
+    n_accepted[b] = n;
+    for (int32_t i = 0; i < n; ++i) ob[i] = xb[i];
+    ob[n] = fresh;
+    if (near) near[b] |= nearbits;
+}
+
+template <class F>
+void for_rows(int32_t B, int32_t n_threads, F f) {
+    n_threads = std::max(1, std::min(n_threads, B));
+    if (n_threads == 1) {
+        for (int32_t b = 0; b < B; ++b) f(b);
+        return;
+    }
+    std::vector<std::thread> pool;
+    for (int32_t t = 0; t < n_threads; ++t)
+        pool.emplace_back([=]() {
+            for (int32_t b = t; b < B; b += n_threads) f(b);
+        });
+    for (auto& th : pool) th.join();
+}
+
+bool batch_ok(const oracle_batch* bt, bool need_target) {
+    if (!bt || bt->B < 0 || bt->gamma_max < 1 || bt->V < 1) return false;
+    if (bt->dtype != ORACLE_DT_F32 && bt->dtype != ORACLE_DT_BF16) return false;
+    if (bt->B > 0 && !bt->draft) return false;
+    if (need_target && bt->B > 0 && (!bt->target || !bt->draft_tokens || !bt->uniforms)) return false;
+    return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int oracle_softmax_row(const void* row, int32_t dtype, int32_t V, double T, double* prob) {
+    return softmax_row(RowRef{row, dtype, 0}, V, T, prob) ? 0 : ORACLE_ROW_NONFINITE;
+}
+
+double oracle_entropy_nats(const double* prob, int32_t V) { return entropy_nats(prob, V); }
+
+int32_t oracle_inverse_cdf(const double* w, int32_t V, double u, int32_t* near_boundary) {
+    return inverse_cdf(w, V, u, near_boundary);
+}
+
+int32_t oracle_argmax_row(const void* row, int32_t dtype, int32_t V) {
+    return argmax_row(RowRef{row, dtype, 0}, V);
+}
+
+int oracle_signals(const oracle_batch* bt, double* H, double* C, double* feat, int32_t* row_status) {
+    if (!batch_ok(bt, false)) return 1;
+    if (row_status) std::fill(row_status, row_status + bt->B, 0);
+    for_rows(bt->B, bt->n_threads, [&](int32_t b) { signals_row(bt, b, H, C, feat, row_status); });
+    return 0;
+}
+
+int oracle_select_gamma(int32_t B, const double* feat, const float* comp, const oracle_mlp* mlp,
+                        double* scores, int32_t* gamma_next, int32_t* near) {
+    if (B < 0 || !mlp || !feat || mlp->n_out < 1 || mlp->n_out > 8 || mlp->n_hidden < 1 ||
+        mlp->n_in < 4)
+        return 1;
+    const int32_t n_comp = mlp->n_in - (mlp->feature_layout == 0 ? 3 : 4);
+    for (int32_t b = 0; b < B; ++b)
+        select_gamma_row(feat + static_cast<int64_t>(b) * 4,
+                         comp ? comp + static_cast<int64_t>(b) * n_comp : nullptr, mlp,
+                         scores ? scores + static_cast<int64_t>(b) * mlp->n_out : nullptr,
+                         gamma_next ? gamma_next + b : nullptr, near ? near + b : nullptr);
+    return 0;
+}
+
+int oracle_verify(const oracle_batch* bt, int32_t* n_accepted, int32_t* out_tokens,
+                  int32_t* row_status, int32_t* near) {
+    if (!batch_ok(bt, true) || !n_accepted || !out_tokens) return 1;
+    if (row_status) std::fill(row_status, row_status + bt->B, 0);
+    if (near) std::fill(near, near + bt->B, 0);
+    for_rows(bt->B, bt->n_threads,
+             [&](int32_t b) { verify_row(bt, b, n_accepted, out_tokens, row_status, near); });
+    return 0;
+}
+
+int oracle_step(const oracle_batch* bt, const float* comp, const oracle_mlp* mlp, double* H,
+                double* C, double* feat, double* scores, int32_t* gamma_next,
+                int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status, int32_t* near) {
+    if (!batch_ok(bt, true) || !mlp || !feat || !n_accepted || !out_tokens || !row_status) return 1;
+    std::fill(row_status, row_status + bt->B, 0);
+    if (near) std::fill(near, near + bt->B, 0);
+    const int32_t n_comp = mlp->n_in - (mlp->feature_layout == 0 ? 3 : 4);
+    for_rows(bt->B, bt->n_threads, [&](int32_t b) {
+        signals_row(bt, b, H, C, feat, row_status);
+        verify_row(bt, b, n_accepted, out_tokens, row_status, near);
+        double* sb = scores ? scores + static_cast<int64_t>(b) * mlp->n_out : nullptr;
+        if (row_status[b]) {
+            /* a flagged row takes no decision */
+            if (sb) std::fill(sb, sb + mlp->n_out, 0.0);
+            if (gamma_next) gamma_next[b] = 0;
+            double* fb = feat + static_cast<int64_t>(b) * 4;
+            std::fill(fb, fb + 4, 0.0);
+            if (H) std::fill(H + static_cast<int64_t>(b) * bt->gamma_max,
+                             H + static_cast<int64_t>(b + 1) * bt->gamma_max, 0.0);
+            if (C) std::fill(C + static_cast<int64_t>(b) * bt->gamma_max,
+                             C + static_cast<int64_t>(b + 1) * bt->gamma_max, 0.0);
+            return;
+        }
+        select_gamma_row(feat + static_cast<int64_t>(b) * 4,
+                         comp ? comp + static_cast<int64_t>(b) * n_comp : nullptr, mlp, sb,
+                         gamma_next ? gamma_next + b : nullptr, near ? near + b : nullptr);
+    });
+    return 0;
+}
+
+}  // extern "C"
