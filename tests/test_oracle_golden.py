@@ -33,6 +33,7 @@ def test_closed_form_case(kind, V, arg, bits, H, c):
     elif kind == "subset":
         x[np.arange(arg) * 7] = -1.0
     r = oracle.signals(oracle.Batch(draft=x[None, None, :], entropy_in_bits=bool(bits)))
-    tol = 1e-7 if kind == "twopoint_ln3" else 1e-13
+    # sequential double sums over V terms carry about V * 1e-16 of rounding
+    tol = 1e-7 if kind == "twopoint_ln3" else max(1e-13, V * 2e-15)
     assert r["H"][0, 0] == pytest.approx(H, rel=tol, abs=1e-15)
     assert r["C"][0, 0] == pytest.approx(c, rel=tol)
