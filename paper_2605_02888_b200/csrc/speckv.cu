@@ -1,0 +1,245 @@
+// Host side of libspeckv: argument checks, workspace plan and kernel launches behind the
+// C ABI declared in include/speckv.h.  No allocation, no synchronisation, no global state.
+#include "speckv.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdint>
+
+#include "speckv_kernels.cuh"
+
+namespace {
+
+using namespace speckv;
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct Plan {
+    int J_full;      // logit rows per batch row with verification: 2*G + 1
+    int nvec;        // kVec-element vectors per logit row
+    int nchunk;      // 256-element chunks per logit row
+    int R;           // resample CTAs per batch row
+    int chunks_per_cta;
+    size_t off_tick, off_info, off_part, off_csum, total;
+};
+
+inline int esize(speckv_dtype dt) { return dt == SPECKV_BF16 ? 2 : 4; }
+
+// vocabulary slices per logit row for a sweep over J logit rows per batch row
+int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
+    const int nvec = (V + kVec - 1) / kVec;
+    const double row_bytes = static_cast<double>(V) * esize(dt);
+    int ns = static_cast<int>(std::lround(row_bytes / 65536.0));
+    if (ns < 1) ns = 1;
+    // small batches: enough CTAs to put a few on every SM
+    const long long rows = static_cast<long long>(B) * J;
+    const long long want = (1184 + rows - 1) / (rows > 0 ? rows : 1);
+    if (want > ns) ns = static_cast<int>(want > kMaxSplit ? kMaxSplit : want);
+    if (ns > kMaxSplit) ns = kMaxSplit;
+    // at least one vector per thread in a slice
+    int cap = nvec / kThreads;
+    if (cap < 1) cap = 1;
+    if (ns > cap) ns = cap;
+    return ns;
+}
+
+Plan make_plan(const speckv_batch* bt) {
+    Plan p;
+    const size_t B = static_cast<size_t>(bt->B);
+    p.J_full = 2 * bt->gamma_max + 1;
+    p.nvec = (bt->V + kVec - 1) / kVec;
+    p.nchunk = (bt->V + kChunk - 1) / kChunk;
+    p.R = (p.nchunk + 63) / 64;
+    if (p.R > 32) p.R = 32;
+    if (p.R < 1) p.R = 1;
+    p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
+    size_t off = 0;
+    p.off_tick = off; off = align_up(off + 2 * B * sizeof(int));
+    p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
+    p.off_part = off; off = align_up(off + B * p.J_full * kMaxSplit * sizeof(float4));
+    p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
+    p.total = off < kAlign ? kAlign : off;
+    return p;
+}
+
+speckv_status check_batch(const speckv_batch* bt, bool need_target) {
+    if (!bt) return SPECKV_ERR_INVALID_ARG;
+    if (bt->B < 0 || bt->gamma_max < 1 || bt->V < 1) return SPECKV_ERR_INVALID_ARG;
+    if (bt->dtype != SPECKV_F32 && bt->dtype != SPECKV_BF16) return SPECKV_ERR_UNSUPPORTED;
+    if (bt->gamma_max > SPECKV_MAX_GAMMA) return SPECKV_ERR_UNSUPPORTED;
+    if (bt->V > (1 << 30) || bt->B > (1 << 24)) return SPECKV_ERR_UNSUPPORTED;
+    if (bt->B == 0) return SPECKV_OK;
+    if (!bt->draft_logits) return SPECKV_ERR_INVALID_ARG;
+    // a stride of 0 broadcasts one row; anything else must step over whole rows
+    auto stride_ok = [&](int64_t s) { return s == 0 || s >= bt->V; };
+    if (!stride_ok(bt->draft_stride_b) || !stride_ok(bt->draft_stride_pos)) return SPECKV_ERR_INVALID_ARG;
+    if (need_target) {
+        if (!bt->target_logits || !bt->draft_tokens || !bt->uniforms) return SPECKV_ERR_INVALID_ARG;
+        if (!stride_ok(bt->target_stride_b) || !stride_ok(bt->target_stride_pos)) return SPECKV_ERR_INVALID_ARG;
+    }
+    if (!(bt->temperature) && !(bt->temperature_scalar >= 0.f)) return SPECKV_ERR_INVALID_ARG;
+    return SPECKV_OK;
+}
+
+speckv_status check_mlp(const speckv_mlp* m) {
+    if (!m || !m->W1 || !m->b1 || !m->W2 || !m->b2) return SPECKV_ERR_INVALID_ARG;
+    if (m->n_hidden < 1 || m->n_out < 1 || m->n_in < 1) return SPECKV_ERR_INVALID_ARG;
+    if (m->n_hidden > SPECKV_MAX_HIDDEN || m->n_out > 8 || m->n_in > 8) return SPECKV_ERR_UNSUPPORTED;
+    if (m->feature_layout != 0 && m->feature_layout != 1) return SPECKV_ERR_INVALID_ARG;
+    if (m->score_transform != 0 && m->score_transform != 1) return SPECKV_ERR_INVALID_ARG;
+    if (m->n_in < (m->feature_layout == 0 ? 3 : 4)) return SPECKV_ERR_INVALID_ARG;
+    return SPECKV_OK;
+}
+
+bool rows_aligned(const void* base, int64_t sb, int64_t sp, int es) {
+    return (reinterpret_cast<uintptr_t>(base) % 16 == 0) && ((sb * es) % 16 == 0) && ((sp * es) % 16 == 0);
+}
+
+void fill_mlp(KParams& P, const speckv_mlp* m, const float* comp) {
+    P.n_in = m->n_in; P.n_hidden = m->n_hidden; P.n_out = m->n_out;
+    P.layout = m->feature_layout; P.transform = m->score_transform;
+    P.n_comp = m->n_in - (m->feature_layout == 0 ? 3 : 4);
+    P.W1 = m->W1; P.b1 = m->b1; P.W2 = m->W2; P.b2 = m->b2; P.comp = comp;
+    for (int j = 0; j < 8; ++j) P.gch[j] = m->gamma_choices[j];
+}
+
+template <typename T, bool ALIGNED>
+cudaError_t launch_all(const KParams& P, cudaStream_t st) {
+    constexpr int U = sizeof(T) == 2 ? 4 : 2;
+    const long long grid = static_cast<long long>(P.B) * P.J * P.nsplit;
+    sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (P.mode & MODE_VERIFY) {
+        resample_kernel<T, ALIGNED><<<dim3(P.B, P.R), kThreads, 0, st>>>(P);
+        e = cudaGetLastError();
+    }
+    return e;
+}
+
+// Shared driver of signals / verify / step.
+speckv_status run(const speckv_batch* bt, int mode, const float* comp, const speckv_mlp* mlp, float* H,
+                  float* C, float* feat, float* scores, int32_t* gamma_next, int32_t* n_accepted,
+                  int32_t* out_tokens, int32_t* row_status, void* ws, size_t ws_bytes, void* stream) {
+    const bool verify = (mode & MODE_VERIFY) != 0;
+    speckv_status st = check_batch(bt, verify);
+    if (st != SPECKV_OK) return st;
+    if (mode & MODE_MLP) {
+        st = check_mlp(mlp);
+        if (st != SPECKV_OK) return st;
+        if (!gamma_next || !feat) return SPECKV_ERR_INVALID_ARG;
+    }
+    if (verify && (!n_accepted || !out_tokens)) return SPECKV_ERR_INVALID_ARG;
+    if (bt->B == 0) return SPECKV_OK;
+    const Plan pl = make_plan(bt);
+    if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SPECKV_ERR_INVALID_ARG;
+    if (ws_bytes < pl.total) return SPECKV_ERR_WORKSPACE;
+
+    KParams P{};
+    P.B = bt->B; P.G = bt->gamma_max; P.V = bt->V;
+    P.J = verify ? pl.J_full : bt->gamma_max;
+    P.nsplit = choose_nsplit(P.B, P.J, P.V, bt->dtype);
+    P.nvec = pl.nvec;
+    P.per_split = (pl.nvec + P.nsplit - 1) / P.nsplit;
+    P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
+    P.mode = mode; P.bits = bt->entropy_in_bits ? 1 : 0;
+    P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
+    P.t = bt->target_logits; P.tsb = bt->target_stride_b; P.tsp = bt->target_stride_pos;
+    P.tok = bt->draft_tokens; P.gamma = bt->gamma; P.temp = bt->temperature;
+    P.temp_scalar = bt->temperature_scalar; P.u = bt->uniforms;
+    if (mode & MODE_MLP) fill_mlp(P, mlp, comp);
+    P.H = H; P.C = C; P.feat = feat; P.scores = scores; P.gamma_next = gamma_next;
+    P.n_acc = n_accepted; P.out_tok = out_tokens; P.status = row_status;
+    char* w = static_cast<char*>(ws);
+    P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
+    P.tick2 = P.tick1 + P.B;
+    P.info = reinterpret_cast<RowInfo*>(w + pl.off_info);
+    P.part = reinterpret_cast<float4*>(w + pl.off_part);
+    P.csum = reinterpret_cast<float*>(w + pl.off_csum);
+
+    if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(P.tick1, 0, 2 * static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess)
+        return SPECKV_ERR_CUDA;
+
+    const int es = esize(bt->dtype);
+    bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
+    if (verify) aligned = aligned && rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
+
+    cudaError_t e;
+    if (bt->dtype == SPECKV_BF16)
+        e = aligned ? launch_all<__nv_bfloat16, true>(P, cs) : launch_all<__nv_bfloat16, false>(P, cs);
+    else
+        e = aligned ? launch_all<float, true>(P, cs) : launch_all<float, false>(P, cs);
+    return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+speckv_status speckv_workspace_size(const speckv_batch* batch, size_t* bytes) {
+    if (!bytes) return SPECKV_ERR_INVALID_ARG;
+    if (!batch || batch->B < 0 || batch->gamma_max < 1 || batch->V < 1) return SPECKV_ERR_INVALID_ARG;
+    if (batch->gamma_max > SPECKV_MAX_GAMMA || batch->V > (1 << 30) || batch->B > (1 << 24))
+        return SPECKV_ERR_UNSUPPORTED;
+    *bytes = make_plan(batch).total;
+    return SPECKV_OK;
+}
+
+speckv_status speckv_signals(const speckv_batch* batch, float* H, float* C, float* feat,
+                             int32_t* row_status, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+    return run(batch, MODE_SIGNALS, nullptr, nullptr, H, C, feat, nullptr, nullptr, nullptr, nullptr,
+               row_status, workspace, workspace_bytes, cuda_stream);
+}
+
+speckv_status speckv_select_gamma(int32_t B, const float* feat, const float* comp,
+                                  const speckv_mlp* mlp, float* scores, int32_t* gamma_next,
+                                  void* cuda_stream) {
+    if (B < 0) return SPECKV_ERR_INVALID_ARG;
+    speckv_status st = check_mlp(mlp);
+    if (st != SPECKV_OK) return st;
+    if (B == 0) return SPECKV_OK;
+    if (!feat || !gamma_next) return SPECKV_ERR_INVALID_ARG;
+    KParams P{};
+    P.B = B;
+    fill_mlp(P, mlp, comp);
+    P.scores = scores; P.gamma_next = gamma_next;
+    const int grid = (B + kWarps - 1) / kWarps;
+    select_gamma_kernel<<<grid, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(P, feat);
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
+speckv_status speckv_verify(const speckv_batch* batch, int32_t* n_accepted, int32_t* out_tokens,
+                            int32_t* row_status, void* workspace, size_t workspace_bytes,
+                            void* cuda_stream) {
+    return run(batch, MODE_VERIFY, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr,
+               n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream);
+}
+
+speckv_status speckv_step(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
+                          float* H, float* C, float* feat, float* scores, int32_t* gamma_next,
+                          int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return run(batch, MODE_SIGNALS | MODE_VERIFY | MODE_MLP, comp, mlp, H, C, feat, scores, gamma_next,
+               n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream);
+}
+
+const char* speckv_status_string(speckv_status s) {
+    switch (s) {
+        case SPECKV_OK: return "ok";
+        case SPECKV_ERR_INVALID_ARG: return "invalid argument";
+        case SPECKV_ERR_UNSUPPORTED: return "unsupported size or type";
+        case SPECKV_ERR_WORKSPACE: return "workspace too small";
+        case SPECKV_ERR_CUDA: return "CUDA launch failed";
+    }
+    return "unknown status";
+}
+
+int speckv_version(void) { return 100; }
+
+}  // extern "C"
