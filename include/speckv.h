@@ -132,6 +132,17 @@ speckv_status speckv_step(const speckv_batch* batch, const float* comp, const sp
                           int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* Measurement aid: speckv_step with three caller-created CUDA events (cudaEvent_t passed as
+ * void*) recorded on the stream before the sweep kernel, between the sweep and the resample
+ * kernel, and after the resample kernel, so that a benchmark can time the dominant kernel
+ * alone.  Results are identical to speckv_step.  Any event may be NULL.                   */
+speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
+                                   float* H, float* C, float* feat, float* scores,
+                                   int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens,
+                                   int32_t* row_status, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream, void* ev_before_sweep, void* ev_after_sweep,
+                                   void* ev_after_resample);
+
 const char* speckv_status_string(speckv_status s);
 int speckv_version(void);
 

@@ -21,7 +21,7 @@ F32, BF16 = 0, 1
 ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE, ROW_TIMEOUT = 0, 1, 2, 4, 8, 16
 
 EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_select_gamma", "speckv_verify",
-           "speckv_step", "speckv_status_string", "speckv_version")
+           "speckv_step", "speckv_step_profiled", "speckv_status_string", "speckv_version")
 
 
 class SpeckvError(RuntimeError):
@@ -74,6 +74,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_verify.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, sz, vp]
     L.speckv_step.restype = C.c_int
     L.speckv_step.argtypes = [C.POINTER(_CBatch), vp, C.POINTER(_CMlp)] + [vp] * 8 + [vp, sz, vp]
+    L.speckv_step_profiled.restype = C.c_int
+    L.speckv_step_profiled.argtypes = L.speckv_step.argtypes + [vp, vp, vp]
     L.speckv_status_string.restype = C.c_char_p
     L.speckv_status_string.argtypes = [C.c_int]
     L.speckv_version.restype = C.c_int
@@ -293,18 +295,29 @@ def speckv_verify(batch: Batch, out: Optional[StepOutputs] = None):
     return dict(n_accepted=o.n_accepted, out_tokens=o.out_tokens, row_status=o.row_status)
 
 
-def speckv_step(batch: Batch, comp: Optional[torch.Tensor], mlp: Mlp, out: Optional[StepOutputs] = None):
-    """Fused step: signals + controller + verification.  Returns the StepOutputs tensors."""
+def speckv_step(batch: Batch, comp: Optional[torch.Tensor], mlp: Mlp, out: Optional[StepOutputs] = None,
+                events: Optional[tuple] = None):
+    """Fused step: signals + controller + verification.  Returns the StepOutputs tensors.
+    `events`: optional (before_sweep, after_sweep, after_resample) torch.cuda.Event objects
+    (created with enable_timing=True); they are recorded around the two kernels."""
     L = load_library()
     c = batch._c()
     m = mlp._c()
     o = out or StepOutputs.allocate(batch, mlp.n_out)
     dev = batch.draft_logits.device
+    args = [C.byref(c), _dev_ptr(comp, torch.float32, "comp"), C.byref(m), _ptr(o.H), _ptr(o.C),
+            _ptr(o.feat), _ptr(o.scores), _ptr(o.gamma_next), _ptr(o.n_accepted),
+            _ptr(o.out_tokens), _ptr(o.row_status), _ptr(o.workspace), o.workspace.numel(), _stream(dev)]
     with torch.cuda.device(dev):
-        rc = L.speckv_step(C.byref(c), _dev_ptr(comp, torch.float32, "comp"), C.byref(m), _ptr(o.H), _ptr(o.C),
-                           _ptr(o.feat), _ptr(o.scores), _ptr(o.gamma_next), _ptr(o.n_accepted),
-                           _ptr(o.out_tokens), _ptr(o.row_status), _ptr(o.workspace), o.workspace.numel(),
-                           _stream(dev))
+        if events is None:
+            rc = L.speckv_step(*args)
+        else:
+            evs = []
+            for e in events:
+                if e is not None and not e.cuda_event:  # torch creates the event lazily on first record
+                    e.record(torch.cuda.current_stream(dev))
+                evs.append(None if e is None else e.cuda_event)
+            rc = L.speckv_step_profiled(*args, *evs)
     if rc != OK:
         raise SpeckvError(rc, "speckv_step")
     return o.as_dict()

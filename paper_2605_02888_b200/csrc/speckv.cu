@@ -13,6 +13,9 @@ namespace {
 
 using namespace speckv;
 
+#ifndef SPECKV_SLICE_BYTES
+#define SPECKV_SLICE_BYTES 262144 // bytes of one logit row that one sweep CTA streams
+#endif
 constexpr size_t kAlign = 256;
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -31,7 +34,7 @@ inline int esize(speckv_dtype dt) { return dt == SPECKV_BF16 ? 2 : 4; }
 int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
     const int nvec = (V + kVec - 1) / kVec;
     const double row_bytes = static_cast<double>(V) * esize(dt);
-    int ns = static_cast<int>(std::lround(row_bytes / 65536.0));
+    int ns = static_cast<int>(std::lround(row_bytes / static_cast<double>(SPECKV_SLICE_BYTES)));
     if (ns < 1) ns = 1;
     // small batches: enough CTAs to put a few on every SM
     const long long rows = static_cast<long long>(B) * J;
@@ -105,24 +108,32 @@ void fill_mlp(KParams& P, const speckv_mlp* m, const float* comp) {
     for (int j = 0; j < 8; ++j) P.gch[j] = m->gamma_choices[j];
 }
 
+struct Events {  // optional timing events around the two kernels
+    cudaEvent_t before_sweep = nullptr, after_sweep = nullptr, after_resample = nullptr;
+};
+
 template <typename T, bool ALIGNED>
-cudaError_t launch_all(const KParams& P, cudaStream_t st) {
+cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev) {
     constexpr int U = sizeof(T) == 2 ? 4 : 2;
     const long long grid = static_cast<long long>(P.B) * P.J * P.nsplit;
+    if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
     sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
     if (P.mode & MODE_VERIFY) {
         resample_kernel<T, ALIGNED><<<dim3(P.B, P.R), kThreads, 0, st>>>(P);
         e = cudaGetLastError();
     }
+    if (ev.after_resample) cudaEventRecord(ev.after_resample, st);
     return e;
 }
 
 // Shared driver of signals / verify / step.
 speckv_status run(const speckv_batch* bt, int mode, const float* comp, const speckv_mlp* mlp, float* H,
                   float* C, float* feat, float* scores, int32_t* gamma_next, int32_t* n_accepted,
-                  int32_t* out_tokens, int32_t* row_status, void* ws, size_t ws_bytes, void* stream) {
+                  int32_t* out_tokens, int32_t* row_status, void* ws, size_t ws_bytes, void* stream,
+                  const Events& ev = Events()) {
     const bool verify = (mode & MODE_VERIFY) != 0;
     speckv_status st = check_batch(bt, verify);
     if (st != SPECKV_OK) return st;
@@ -171,9 +182,9 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
 
     cudaError_t e;
     if (bt->dtype == SPECKV_BF16)
-        e = aligned ? launch_all<__nv_bfloat16, true>(P, cs) : launch_all<__nv_bfloat16, false>(P, cs);
+        e = aligned ? launch_all<__nv_bfloat16, true>(P, cs, ev) : launch_all<__nv_bfloat16, false>(P, cs, ev);
     else
-        e = aligned ? launch_all<float, true>(P, cs) : launch_all<float, false>(P, cs);
+        e = aligned ? launch_all<float, true>(P, cs, ev) : launch_all<float, false>(P, cs, ev);
     return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 
@@ -227,6 +238,20 @@ speckv_status speckv_step(const speckv_batch* batch, const float* comp, const sp
                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return run(batch, MODE_SIGNALS | MODE_VERIFY | MODE_MLP, comp, mlp, H, C, feat, scores, gamma_next,
                n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream);
+}
+
+speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
+                                   float* H, float* C, float* feat, float* scores,
+                                   int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens,
+                                   int32_t* row_status, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream, void* ev_before_sweep, void* ev_after_sweep,
+                                   void* ev_after_resample) {
+    Events ev;
+    ev.before_sweep = static_cast<cudaEvent_t>(ev_before_sweep);
+    ev.after_sweep = static_cast<cudaEvent_t>(ev_after_sweep);
+    ev.after_resample = static_cast<cudaEvent_t>(ev_after_resample);
+    return run(batch, MODE_SIGNALS | MODE_VERIFY | MODE_MLP, comp, mlp, H, C, feat, scores, gamma_next,
+               n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream, ev);
 }
 
 const char* speckv_status_string(speckv_status s) {

@@ -370,29 +370,83 @@ __device__ __forceinline__ float4 shfl_xor4(float4 v, int mask) {
 }
 
 // ----------------------------------------------------------------------------------------
+// Warp-level merge of the 32 per-thread partials (result valid in every lane).
+// DRAFT / TARGET: bring every lane to the warp-wide reference, then plain sums.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sumf(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_maxf(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+template <int PATH>
+__device__ __forceinline__ float4 warp_merge(float4 p, float scale) {
+    if constexpr (PATH == PATH_DRAFT) {
+        const float M = warp_maxf(p.x);
+        if (p.x != M) {  // this lane's maximum is not the warp's: its count joins the scaled sum
+            const float dm = p.x - M, f = ex2f(dm * scale), za = p.y + p.z;
+            p.w = fmaf(dm, za, p.w) * f;
+            p.z = za * f;
+            p.y = 0.f;
+        }
+        return make_float4(M, warp_sumf(p.y), warp_sumf(p.z), warp_sumf(p.w));
+    } else if constexpr (PATH == PATH_TARGET) {
+        const float R = warp_maxf(p.x);
+        return make_float4(R, warp_sumf(p.y * ex2f(p.x - R)), 0.f, 0.f);
+    } else {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) p = merge_argmax(p, shfl_xor4(p, o));
+        return p;
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ Raw<T> ld_vec(const T* p) {
+    Raw<T> r;
+    if constexpr (sizeof(T) == 2) {
+        r.a = ldg_stream(p);
+    } else {
+        r.a = ldg_stream(p);
+        r.b = ldg_stream(p + 4);
+    }
+    return r;
+}
+
+// ----------------------------------------------------------------------------------------
 // One CTA sweeps elements [lo, hi) of one logit row and returns the merged partial in
-// thread 0.  U vectors per thread are kept in flight.
+// thread 0.  Thread t owns vectors t, t+256, ... of the slice; U of them are in flight.
 // ----------------------------------------------------------------------------------------
 template <typename T, bool ALIGNED, int PATH, int U>
-__device__ __forceinline__ float4 sweep_slice(const T* row, int lo, int hi, float scale, float4* sh_part) {
+__device__ __forceinline__ float4 sweep_slice(const T* __restrict__ row, int lo, int hi, float scale,
+                                              float4* sh_part) {
     const int tid = threadIdx.x;
     const float pad = (PATH == PATH_DRAFT) ? kFloor : __int_as_float(0xff800000);
-    const int nv = (hi - lo + kVec - 1) / kVec;           // vectors in the slice
-    const int niter = (nv + kThreads - 1) / kThreads;      // steps per thread (uniform)
+    constexpr int kStride = kThreads * kVec;               // elements between a thread's vectors
+    const int nv = (hi - lo + kVec - 1) / kVec;             // vectors in the slice (last may be ragged)
+    const int my_n = (nv > tid) ? (nv - tid + kThreads - 1) / kThreads : 0;
+    // vectors this thread takes through the unguarded 16-byte path
+    int n_main = my_n;
+    if (!ALIGNED) n_main = 0;
+    else if (my_n > 0 && lo + (tid + (my_n - 1) * kThreads) * kVec + kVec > hi) n_main = my_n - 1;
+    const T* p = row + lo + tid * kVec;
 
     Raw<T> buf[U];
 #pragma unroll
-    for (int k = 0; k < U; ++k) {
-        int e0 = lo + (k * kThreads + tid) * kVec;
-        buf[k] = (k < niter) ? load_raw<T, ALIGNED>(row, e0, hi, pad) : raw_fill<T>(pad);
-    }
-    // warm start: the CTA-wide maximum of every thread's first vector
-    float m0 = raw_max(buf[0]);
-    // a first vector holding NaN / +inf / only -inf contributes the floor; its owner meets the
-    // offending element again in its own state and flags it there
+    for (int k = 0; k < U; ++k) buf[k] = (k < n_main) ? ld_vec<T>(p + k * kStride) : raw_fill<T>(pad);
+    Raw<T> first = buf[0];
+    if (n_main == 0 && my_n > 0) first = load_raw<T, false>(row, lo + tid * kVec, hi, pad);
+
+    // warm start: the CTA-wide maximum of every thread's first vector.  A first vector holding
+    // NaN / +inf / only -inf contributes the floor; its owner meets the offending element again
+    // in its own state and flags it there.
+    float m0 = raw_max(first);
     if (!(m0 >= kFloor && m0 < __int_as_float(0x7f800000))) m0 = kFloor;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, o));
+    m0 = warp_maxf(m0);
     __shared__ float sh_m0[kWarps];
     if ((tid & 31) == 0) sh_m0[tid >> 5] = m0;
     __syncthreads();
@@ -405,39 +459,42 @@ __device__ __forceinline__ float4 sweep_slice(const T* row, int lo, int hi, floa
     else if constexpr (PATH == PATH_TARGET) ts.init(m0, scale);
     else as.init(m0);
 
-    for (int it = 0; it < niter; it += U) {
+    auto process = [&](const Raw<T>& v, int idx) {
+        if constexpr (PATH == PATH_DRAFT) ds.template step<T>(v, scale);
+        else if constexpr (PATH == PATH_TARGET) ts.template step<T>(v, scale);
+        else as.template step<T>(v, lo + (tid + idx * kThreads) * kVec);
+    };
+
+    int i = 0;
+    for (; i + U <= n_main; i += U) {
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            Raw<T> cur = buf[k];
-            const int e_cur = lo + ((it + k) * kThreads + tid) * kVec;
-            const int itn = it + k + U;
-            if (itn < niter) buf[k] = load_raw<T, ALIGNED>(row, lo + (itn * kThreads + tid) * kVec, hi, pad);
-            if (it + k < niter) {
-                if constexpr (PATH == PATH_DRAFT) {
-                    if (it + k == 0) ds.template slow<T>(cur, scale);  // owns its share of the warm-start maximum
-                    else ds.template step<T>(cur, scale);
-                } else if constexpr (PATH == PATH_TARGET) {
-                    ts.template step<T>(cur, scale);
-                } else {
-                    as.template step<T>(cur, e_cur);
-                }
-            }
+            const Raw<T> cur = buf[k];
+            const int nx = i + U + k;
+            if (nx < n_main) buf[k] = ld_vec<T>(p + nx * kStride);
+            process(cur, i + k);
         }
     }
-
-    float4 p;
-    if constexpr (PATH == PATH_DRAFT) p = ds.partial();
-    else if constexpr (PATH == PATH_TARGET) p = ts.partial();
-    else p = as.partial();
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) p = merge_any<PATH>(p, shfl_xor4(p, o), scale);
-    if ((tid & 31) == 0) sh_part[tid >> 5] = p;
+    for (int k = 0; k < U; ++k)
+        if (i + k < n_main) process(buf[k], i + k);
+    // vectors that need the guarded element-wise load: a ragged last vector, or every vector
+    // of a row that is not 16-byte aligned
+    for (int j = n_main; j < my_n; ++j)
+        process(load_raw<T, false>(row, lo + (tid + j * kThreads) * kVec, hi, pad), j);
+
+    float4 part;
+    if constexpr (PATH == PATH_DRAFT) part = ds.partial();
+    else if constexpr (PATH == PATH_TARGET) part = ts.partial();
+    else part = as.partial();
+    part = warp_merge<PATH>(part, scale);
+    if ((tid & 31) == 0) sh_part[tid >> 5] = part;
     __syncthreads();
     if (tid == 0) {
 #pragma unroll
-        for (int w = 1; w < kWarps; ++w) p = merge_any<PATH>(p, sh_part[w], scale);
+        for (int w = 1; w < kWarps; ++w) part = merge_any<PATH>(part, sh_part[w], scale);
     }
-    return p;
+    return part;
 }
 
 // ----------------------------------------------------------------------------------------
@@ -657,7 +714,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
 // Sweep kernel
 // ----------------------------------------------------------------------------------------
 template <typename T, bool ALIGNED, int U>
-__global__ void __launch_bounds__(kThreads, 4) sweep_kernel(const KParams P) {
+__global__ void __launch_bounds__(kThreads, 4) sweep_kernel(const __grid_constant__ KParams P) {
     __shared__ float4 sh_part[kWarps];
     __shared__ int sh_last;
 
@@ -810,7 +867,7 @@ __device__ __forceinline__ double rs_total(const float* csum, int nchunk, int pe
 }
 
 template <typename T, bool ALIGNED>
-__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const KParams P) {
+__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ KParams P) {
     __shared__ int sh_flag;
     __shared__ int sh_empty;
     const int b = blockIdx.x;  // batch row; blockIdx.y = which share of the row's chunks
@@ -927,7 +984,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const KParams P) 
 // ----------------------------------------------------------------------------------------
 // Stand-alone controller: one warp per row.
 // ----------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) select_gamma_kernel(const KParams P, const float* feat_in) {
+__global__ void __launch_bounds__(kThreads) select_gamma_kernel(const __grid_constant__ KParams P, const float* feat_in) {
     const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (b >= P.B) return;
     double f4[4];
