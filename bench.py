@@ -163,6 +163,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="b256")
     ap.add_argument("--rows", type=int, default=None, help="override the workload's batch rows (profiling captures)")
+    ap.add_argument("--lib", default=None, help="path of a libspeckv.so build to load instead of the in-tree one")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -183,6 +184,9 @@ def main():
 
     import torch
     import paper_2605_02888_b200 as speckv
+    if args.lib:
+        from paper_2605_02888_b200 import binding
+        binding._lib = binding.load_library(args.lib)
 
     def gpu_batch(s):
         return speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],

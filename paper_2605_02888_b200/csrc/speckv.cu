@@ -114,7 +114,7 @@ struct Events {  // optional timing events around the two kernels
 
 template <typename T, bool ALIGNED>
 cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev) {
-    constexpr int U = sizeof(T) == 2 ? 4 : 2;
+    constexpr int U = sizeof(T) == 2 ? SPECKV_U : (SPECKV_U + 1) / 2;
     const long long grid = static_cast<long long>(P.B) * P.J * P.nsplit;
     if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
     sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);

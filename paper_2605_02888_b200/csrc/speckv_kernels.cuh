@@ -23,6 +23,21 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kVec = 8;                 // elements per lane per step
 constexpr int kChunk = 32 * kVec;       // one warp step = one inverse-CDF chunk (256 elements)
 constexpr int kMaxSplit = 32;
+#ifndef SPECKV_WARP_RANGES
+#define SPECKV_WARP_RANGES 0  // 1: each warp streams its own contiguous range; 0: the CTA's threads interleave
+#endif
+#ifndef SPECKV_PACKED
+#define SPECKV_PACKED 1       // 1: f32x2 packed arithmetic in the sweep; 0: scalar fp32
+#endif
+#ifndef SPECKV_SYNC_WARM
+#define SPECKV_SYNC_WARM 1    // 1: CTA barrier before reading the other warps' warm-start maxima; 0: read what is there
+#endif
+#ifndef SPECKV_U
+#define SPECKV_U 4            // 16-byte loads in flight per thread (bf16); fp32 uses half as many vector steps
+#endif
+#ifndef SPECKV_MINB
+#define SPECKV_MINB 4         // CTAs per SM the sweep kernel is compiled for
+#endif
 constexpr float kFloor = -1.2676506002282294e30f;  // -2^100: logits below count as -inf
 constexpr uint32_t kFloorBf16x2 = 0xF180F180u;     // -2^100 as two bf16
 constexpr double kLn2 = 0.6931471805599453094;
@@ -68,6 +83,47 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Packed pairs of fp32 (sm_100 f32x2 arithmetic): one instruction works on two elements.
+typedef unsigned long long f2;
+__device__ __forceinline__ f2 pack2(float a, float b) {
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b) {
+    f2 r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 sub2(f2 a, f2 b) {
+    f2 r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 mul2(f2 a, f2 b) {
+    f2 r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) {
+    f2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+__device__ __forceinline__ f2 ex2_2(f2 a) {
+    float x, y;
+    unpack2(a, x, y);
+    return pack2(ex2f(x), ex2f(y));
+}
+__device__ __forceinline__ float hsum2(f2 a) {
+    float x, y;
+    unpack2(a, x, y);
+    return x + y;
+}
+
 __device__ __forceinline__ float max_nan(float a, float b) {  // NaN-propagating max
     float y;
     asm("max.NaN.f32 %0, %1, %2;" : "=f"(y) : "f"(a), "f"(b));
@@ -115,6 +171,18 @@ template <> __device__ __forceinline__ void unpack<float>(const Raw<float>& r, f
     x[2] = __uint_as_float(r.a.z); x[3] = __uint_as_float(r.a.w);
     x[4] = __uint_as_float(r.b.x); x[5] = __uint_as_float(r.b.y);
     x[6] = __uint_as_float(r.b.z); x[7] = __uint_as_float(r.b.w);
+}
+
+// the same kVec elements as four packed pairs
+__device__ __forceinline__ void unpack_pairs(const Raw<__nv_bfloat16>& r, f2 (&x)[4]) {
+    x[0] = pack2(bf_lo(r.a.x), bf_hi(r.a.x)); x[1] = pack2(bf_lo(r.a.y), bf_hi(r.a.y));
+    x[2] = pack2(bf_lo(r.a.z), bf_hi(r.a.z)); x[3] = pack2(bf_lo(r.a.w), bf_hi(r.a.w));
+}
+__device__ __forceinline__ void unpack_pairs(const Raw<float>& r, f2 (&x)[4]) {
+    x[0] = pack2(__uint_as_float(r.a.x), __uint_as_float(r.a.y));
+    x[1] = pack2(__uint_as_float(r.a.z), __uint_as_float(r.a.w));
+    x[2] = pack2(__uint_as_float(r.b.x), __uint_as_float(r.b.y));
+    x[3] = pack2(__uint_as_float(r.b.z), __uint_as_float(r.b.w));
 }
 
 __device__ __forceinline__ float elem_to_float(const __nv_bfloat16* p, long long i) {
@@ -216,9 +284,15 @@ __device__ __forceinline__ void raw_floor(Raw<float>& r) {
 // ARGMAX  a = best value, b = index (bit pattern), c = bad flag (non-zero: NaN / +inf seen).
 // ----------------------------------------------------------------------------------------
 struct DraftState {
-    float m, cnt, z0, z1, s0, s1;
+    float m, cnt;
+    f2 za, zb, sa, sb;  // four running sums each of Zx and S, as two packed pairs
     bool bad;
-    __device__ __forceinline__ void init(float m0) { m = m0; cnt = 0.f; z0 = z1 = s0 = s1 = 0.f; bad = false; }
+    __device__ __forceinline__ void init(float m0) {
+        m = m0; cnt = 0.f; bad = false;
+        za = zb = sa = sb = pack2(0.f, 0.f);
+    }
+    __device__ __forceinline__ float zsum() const { return hsum2(za) + hsum2(zb); }
+    __device__ __forceinline__ float ssum() const { return hsum2(sa) + hsum2(sb); }
 
     template <typename T>
     __device__ __forceinline__ void slow(const Raw<T>& raw, float scale) {
@@ -231,13 +305,13 @@ struct DraftState {
             x[j] = fmaxf(x[j], kFloor);
             vmax = fmaxf(vmax, x[j]);
         }
+        float z = zsum(), sv = ssum();
         if (vmax > m) {  // everything gathered so far moves below the new maximum
             float dm = m - vmax;
             float f = ex2f(dm * scale);
-            float zall = cnt + (z0 + z1);
-            float sall = s0 + s1;
-            z0 = zall * f; z1 = 0.f;
-            s0 = fmaf(dm, zall, sall) * f; s1 = 0.f;
+            float zall = cnt + z;
+            z = zall * f;
+            sv = fmaf(dm, zall, sv) * f;
             cnt = 0.f;
             m = vmax;
         }
@@ -248,31 +322,55 @@ struct DraftState {
             } else {
                 float dx = x[j] - m;
                 float e = ex2f(dx * scale);
-                z0 += e;
-                s0 = fmaf(e, dx, s0);
+                z += e;
+                sv = fmaf(e, dx, sv);
             }
         }
+        za = pack2(z, 0.f); zb = pack2(0.f, 0.f);
+        sa = pack2(sv, 0.f); sb = pack2(0.f, 0.f);
     }
 
     template <typename T>
     __device__ __forceinline__ void step(Raw<T> raw, float scale) {
+#ifdef SPECKV_EXPERIMENT_NOMATH  // measurement only: keeps the loads, drops the arithmetic
+        cnt += __uint_as_float((raw.a.x ^ raw.a.y ^ raw.a.z ^ raw.a.w) & 0x007fffffu);
+        return;
+#endif
         if (raw_exceeds<false>(raw, m)) {  // an element >= m, or a NaN: rare after the warm start
             slow<T>(raw, scale);
             return;
         }
         raw_floor(raw);
-        float x[kVec];
-        unpack<T>(raw, x);
+#if !SPECKV_PACKED
+        {
+            float xs[kVec];
+            unpack<T>(raw, xs);
+            float z0, z1, z2, z3, s0, s1, s2, s3;
+            unpack2(za, z0, z1); unpack2(zb, z2, z3); unpack2(sa, s0, s1); unpack2(sb, s2, s3);
 #pragma unroll
-        for (int j = 0; j < kVec; j += 2) {
-            float d0 = x[j] - m, d1 = x[j + 1] - m;
-            float e0 = ex2f(d0 * scale), e1 = ex2f(d1 * scale);
-            z0 += e0; z1 += e1;
-            s0 = fmaf(e0, d0, s0); s1 = fmaf(e1, d1, s1);
+            for (int j = 0; j < kVec; j += 4) {
+                float d0 = xs[j] - m, d1 = xs[j + 1] - m, d2 = xs[j + 2] - m, d3 = xs[j + 3] - m;
+                float e0 = ex2f(d0 * scale), e1 = ex2f(d1 * scale), e2 = ex2f(d2 * scale), e3 = ex2f(d3 * scale);
+                z0 += e0; z1 += e1; z2 += e2; z3 += e3;
+                s0 = fmaf(e0, d0, s0); s1 = fmaf(e1, d1, s1); s2 = fmaf(e2, d2, s2); s3 = fmaf(e3, d3, s3);
+            }
+            za = pack2(z0, z1); zb = pack2(z2, z3); sa = pack2(s0, s1); sb = pack2(s2, s3);
+            return;
         }
+#endif
+        f2 x[4];
+        unpack_pairs(raw, x);
+        const f2 m2 = pack2(m, m), sc2 = pack2(scale, scale);
+        const f2 d0 = sub2(x[0], m2), d1 = sub2(x[1], m2), d2 = sub2(x[2], m2), d3 = sub2(x[3], m2);
+        const f2 e0 = ex2_2(mul2(d0, sc2)), e1 = ex2_2(mul2(d1, sc2));
+        const f2 e2 = ex2_2(mul2(d2, sc2)), e3 = ex2_2(mul2(d3, sc2));
+        za = add2(za, e0); zb = add2(zb, e1);
+        sa = fma2(e0, d0, sa); sb = fma2(e1, d1, sb);
+        za = add2(za, e2); zb = add2(zb, e3);
+        sa = fma2(e2, d2, sa); sb = fma2(e3, d3, sb);
     }
     __device__ __forceinline__ float4 partial() const {
-        return make_float4(m, bad ? __int_as_float(0x7fc00000) : cnt, z0 + z1, s0 + s1);
+        return make_float4(m, bad ? __int_as_float(0x7fc00000) : cnt, zsum(), ssum());
     }
 };
 
@@ -293,28 +391,54 @@ __device__ __forceinline__ float4 merge_draft(float4 a, float4 b, float scale) {
 }
 
 struct TargetState {
-    float m, r, z0, z1;
-    __device__ __forceinline__ void init(float m0, float scale) { m = m0; r = m0 * scale; z0 = z1 = 0.f; }
+    float m, r;
+    f2 za, zb;
+    __device__ __forceinline__ void init(float m0, float scale) {
+        m = m0; r = m0 * scale;
+        za = zb = pack2(0.f, 0.f);
+    }
     template <typename T>
     __device__ __forceinline__ void step(const Raw<T>& raw, float scale) {
+#ifdef SPECKV_EXPERIMENT_NOMATH
+        r += __uint_as_float((raw.a.x ^ raw.a.y ^ raw.a.z ^ raw.a.w) & 0x007fffffu);
+        return;
+#endif
         if (raw_exceeds<true>(raw, m)) {  // a new maximum (or NaN): move the reference
             float vmax = raw_max(raw);
             if (vmax == vmax) {  // NaN needs no rescale; it poisons Z below
                 float rn = vmax * scale;
                 float f = ex2f(r - rn);
-                z0 = (z0 + z1) * f; z1 = 0.f;
+                za = pack2((hsum2(za) + hsum2(zb)) * f, 0.f);
+                zb = pack2(0.f, 0.f);
                 r = rn; m = vmax;
             }
         }
-        float x[kVec];
-        unpack<T>(raw, x);
+#if !SPECKV_PACKED
+        {
+            float xs[kVec];
+            unpack<T>(raw, xs);
+            float z0, z1, z2, z3;
+            unpack2(za, z0, z1); unpack2(zb, z2, z3);
 #pragma unroll
-        for (int j = 0; j < kVec; j += 2) {
-            z0 += ex2f(fmaf(x[j], scale, -r));
-            z1 += ex2f(fmaf(x[j + 1], scale, -r));
+            for (int j = 0; j < kVec; j += 4) {
+                z0 += ex2f(fmaf(xs[j], scale, -r)); z1 += ex2f(fmaf(xs[j + 1], scale, -r));
+                z2 += ex2f(fmaf(xs[j + 2], scale, -r)); z3 += ex2f(fmaf(xs[j + 3], scale, -r));
+            }
+            za = pack2(z0, z1); zb = pack2(z2, z3);
+            return;
         }
+#endif
+        f2 x[4];
+        unpack_pairs(raw, x);
+        const f2 sc2 = pack2(scale, scale), nr2 = pack2(-r, -r);
+        const f2 e0 = ex2_2(fma2(x[0], sc2, nr2)), e1 = ex2_2(fma2(x[1], sc2, nr2));
+        const f2 e2 = ex2_2(fma2(x[2], sc2, nr2)), e3 = ex2_2(fma2(x[3], sc2, nr2));
+        za = add2(za, e0); zb = add2(zb, e1);
+        za = add2(za, e2); zb = add2(zb, e3);
     }
-    __device__ __forceinline__ float4 partial() const { return make_float4(r, z0 + z1, 0.f, 0.f); }
+    __device__ __forceinline__ float4 partial() const {
+        return make_float4(r, hsum2(za) + hsum2(zb), 0.f, 0.f);
+    }
 };
 
 __device__ __forceinline__ float4 merge_target(float4 a, float4 b) {
@@ -418,41 +542,53 @@ __device__ __forceinline__ Raw<T> ld_vec(const T* p) {
 }
 
 // ----------------------------------------------------------------------------------------
-// One CTA sweeps elements [lo, hi) of one logit row and returns the merged partial in
-// thread 0.  Thread t owns vectors t, t+256, ... of the slice; U of them are in flight.
+// One WARP sweeps elements [lo, hi) of one logit row and returns the merged partial in every
+// lane.  Lane l owns vectors l, l+32, ... of the range; U of them are in flight.  Warps of a
+// CTA never wait for one another.
 // ----------------------------------------------------------------------------------------
-template <typename T, bool ALIGNED, int PATH, int U>
-__device__ __forceinline__ float4 sweep_slice(const T* __restrict__ row, int lo, int hi, float scale,
-                                              float4* sh_part) {
-    const int tid = threadIdx.x;
+template <typename T, bool ALIGNED, int PATH, int U, int STEP>
+__device__ __forceinline__ float4 sweep_warp(const T* __restrict__ row, int lo, int hi, int first, float scale,
+                                             volatile float* sh_m0) {
+    // this thread owns vectors first, first+STEP, ... of the range [lo, hi)
     const float pad = (PATH == PATH_DRAFT) ? kFloor : __int_as_float(0xff800000);
-    constexpr int kStride = kThreads * kVec;               // elements between a thread's vectors
-    const int nv = (hi - lo + kVec - 1) / kVec;             // vectors in the slice (last may be ragged)
-    const int my_n = (nv > tid) ? (nv - tid + kThreads - 1) / kThreads : 0;
+    constexpr int kStride = STEP * kVec;                    // elements between a thread's vectors
+    const int nv = (hi > lo) ? (hi - lo + kVec - 1) / kVec : 0;  // vectors in the range (last may be ragged)
+    const int my_n = (nv > first) ? (nv - first + STEP - 1) / STEP : 0;
     // vectors this thread takes through the unguarded 16-byte path
     int n_main = my_n;
     if (!ALIGNED) n_main = 0;
-    else if (my_n > 0 && lo + (tid + (my_n - 1) * kThreads) * kVec + kVec > hi) n_main = my_n - 1;
-    const T* p = row + lo + tid * kVec;
+    else if (my_n > 0 && lo + (first + (my_n - 1) * STEP) * kVec + kVec > hi) n_main = my_n - 1;
+    const T* p = row + lo + first * kVec;
 
     Raw<T> buf[U];
 #pragma unroll
     for (int k = 0; k < U; ++k) buf[k] = (k < n_main) ? ld_vec<T>(p + k * kStride) : raw_fill<T>(pad);
-    Raw<T> first = buf[0];
-    if (n_main == 0 && my_n > 0) first = load_raw<T, false>(row, lo + tid * kVec, hi, pad);
 
-    // warm start: the CTA-wide maximum of every thread's first vector.  A first vector holding
+    // warm start: the warp-wide maximum of the first U vectors of every lane.  A vector holding
     // NaN / +inf / only -inf contributes the floor; its owner meets the offending element again
     // in its own state and flags it there.
-    float m0 = raw_max(first);
-    if (!(m0 >= kFloor && m0 < __int_as_float(0x7f800000))) m0 = kFloor;
-    m0 = warp_maxf(m0);
-    __shared__ float sh_m0[kWarps];
-    if ((tid & 31) == 0) sh_m0[tid >> 5] = m0;
-    __syncthreads();
-    m0 = sh_m0[0];
+    float m0 = kFloor;
 #pragma unroll
-    for (int w = 1; w < kWarps; ++w) m0 = fmaxf(m0, sh_m0[w]);
+    for (int k = 0; k < U; ++k) {
+        float v = raw_max(buf[k]);
+        if (v >= kFloor && v < __int_as_float(0x7f800000)) m0 = fmaxf(m0, v);
+    }
+    if (n_main == 0 && my_n > 0) {
+        float v = raw_max(load_raw<T, false>(row, lo + first * kVec, hi, pad));
+        if (v >= kFloor && v < __int_as_float(0x7f800000)) m0 = fmaxf(m0, v);
+    }
+    m0 = warp_maxf(m0);
+    // share the warm start across the CTA's warps: publish ours, take what the others have
+    // published so far (slots start at the floor).  Nobody waits; a late warp only costs the
+    // readers a few more trips through the slow path.
+    if ((threadIdx.x & 31) == 0) sh_m0[threadIdx.x >> 5] = m0;
+#if SPECKV_SYNC_WARM
+    __syncthreads();
+#else
+    __syncwarp();
+#endif
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) m0 = fmaxf(m0, sh_m0[w]);
 
     DraftState ds; TargetState ts; ArgmaxState as;
     if constexpr (PATH == PATH_DRAFT) ds.init(m0);
@@ -462,7 +598,7 @@ __device__ __forceinline__ float4 sweep_slice(const T* __restrict__ row, int lo,
     auto process = [&](const Raw<T>& v, int idx) {
         if constexpr (PATH == PATH_DRAFT) ds.template step<T>(v, scale);
         else if constexpr (PATH == PATH_TARGET) ts.template step<T>(v, scale);
-        else as.template step<T>(v, lo + (tid + idx * kThreads) * kVec);
+        else as.template step<T>(v, lo + (first + idx * STEP) * kVec);
     };
 
     int i = 0;
@@ -481,20 +617,13 @@ __device__ __forceinline__ float4 sweep_slice(const T* __restrict__ row, int lo,
     // vectors that need the guarded element-wise load: a ragged last vector, or every vector
     // of a row that is not 16-byte aligned
     for (int j = n_main; j < my_n; ++j)
-        process(load_raw<T, false>(row, lo + (tid + j * kThreads) * kVec, hi, pad), j);
+        process(load_raw<T, false>(row, lo + (first + j * STEP) * kVec, hi, pad), j);
 
     float4 part;
     if constexpr (PATH == PATH_DRAFT) part = ds.partial();
     else if constexpr (PATH == PATH_TARGET) part = ts.partial();
     else part = as.partial();
-    part = warp_merge<PATH>(part, scale);
-    if ((tid & 31) == 0) sh_part[tid >> 5] = part;
-    __syncthreads();
-    if (tid == 0) {
-#pragma unroll
-        for (int w = 1; w < kWarps; ++w) part = merge_any<PATH>(part, sh_part[w], scale);
-    }
-    return part;
+    return warp_merge<PATH>(part, scale);
 }
 
 // ----------------------------------------------------------------------------------------
@@ -714,10 +843,15 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
 // Sweep kernel
 // ----------------------------------------------------------------------------------------
 template <typename T, bool ALIGNED, int U>
-__global__ void __launch_bounds__(kThreads, 4) sweep_kernel(const __grid_constant__ KParams P) {
+__global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __grid_constant__ KParams P) {
     __shared__ float4 sh_part[kWarps];
-    __shared__ int sh_last;
+    __shared__ int sh_count;
+    __shared__ float sh_m0[kWarps];
+    if (threadIdx.x == 0) sh_count = 0;
+    if (threadIdx.x < kWarps) sh_m0[threadIdx.x] = kFloor;
+    __syncthreads();  // before any load is issued
 
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int per_row = P.J * P.nsplit;
     const int b = blockIdx.x / per_row;
     const int rem = blockIdx.x - b * per_row;
@@ -738,121 +872,157 @@ __global__ void __launch_bounds__(kThreads, 4) sweep_kernel(const __grid_constan
     const bool active = row_ok && (is_target ? pos <= gam : pos < gam);
 
     if (active) {
+        // the CTA's slice of the row
         const int v0 = s * P.per_split;
         const int v1 = min(P.nvec, v0 + P.per_split);
+#if SPECKV_WARP_RANGES
+        // one contiguous range per warp (whole warp-steps)
+        constexpr int STEP = 32;
+        const int first = lane;
+        const int per_warp = (((v1 - v0) + kWarps - 1) / kWarps + 31) / 32 * 32;
+        const int wv0 = min(v1, v0 + warp * per_warp);
+        const int wv1 = min(v1, wv0 + per_warp);
+        const int lo = wv0 * kVec;
+        const int hi = min(P.V, wv1 * kVec);
+#else
+        // the CTA's threads interleave over the slice: consecutive warps read consecutive 512 bytes
+        constexpr int STEP = kThreads;
+        const int first = threadIdx.x;
         const int lo = v0 * kVec;
         const int hi = min(P.V, v1 * kVec);
-        float4 part = make_float4(0.f, 0.f, 0.f, 0.f);
+#endif
+        float4 part;
+        int path;
         if (is_target) {
             const T* row = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
                            static_cast<long long>(pos) * P.tsp;
-            if (greedy) part = sweep_slice<T, ALIGNED, PATH_ARGMAX, U>(row, lo, hi, scale, sh_part);
-            else part = sweep_slice<T, ALIGNED, PATH_TARGET, U>(row, lo, hi, scale, sh_part);
+            if (greedy) { part = sweep_warp<T, ALIGNED, PATH_ARGMAX, U, STEP>(row, lo, hi, first, scale, sh_m0); path = PATH_ARGMAX; }
+            else { part = sweep_warp<T, ALIGNED, PATH_TARGET, U, STEP>(row, lo, hi, first, scale, sh_m0); path = PATH_TARGET; }
         } else {
             const T* row = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb +
                            static_cast<long long>(pos) * P.dsp;
-            part = sweep_slice<T, ALIGNED, PATH_DRAFT, U>(row, lo, hi, scale, sh_part);
+            part = sweep_warp<T, ALIGNED, PATH_DRAFT, U, STEP>(row, lo, hi, first, scale, sh_m0);
+            path = PATH_DRAFT;
         }
-        if (threadIdx.x == 0) P.part[static_cast<long long>(blockIdx.x)] = part;
+        // the last warp of the CTA to finish merges the eight warp partials; nobody waits
+        int last = 0;
+        if (lane == 0) {
+            sh_part[warp] = part;
+            __threadfence_block();
+            last = (atomicAdd(&sh_count, 1) == kWarps - 1);
+        }
+        if (!__shfl_sync(0xffffffffu, last, 0)) return;
+        if (lane == 0) {
+            __threadfence_block();
+            const volatile float4* vp = sh_part;
+            float4 acc = make_float4(vp[0].x, vp[0].y, vp[0].z, vp[0].w);
+            for (int w = 1; w < kWarps; ++w) {
+                float4 o = make_float4(vp[w].x, vp[w].y, vp[w].z, vp[w].w);
+                acc = (path == PATH_DRAFT) ? merge_draft(acc, o, scale)
+                    : (path == PATH_TARGET) ? merge_target(acc, o) : merge_argmax(acc, o);
+            }
+            P.part[static_cast<long long>(blockIdx.x)] = acc;
+        }
+    } else if (warp != 0) {
+        return;
     }
 
     // ticket: the last CTA of this batch row runs the row epilogue; nobody waits
-    if (threadIdx.x == 0) {
+    int last_row = 0;
+    if (lane == 0) {
         __threadfence();
-        int old = atomicAdd(P.tick1 + b, 1);
-        sh_last = (old == per_row - 1);
+        last_row = (atomicAdd(P.tick1 + b, 1) == per_row - 1);
     }
-    __syncthreads();
-    if (!sh_last) return;
+    if (!__shfl_sync(0xffffffffu, last_row, 0)) return;
     __threadfence();
-    if (threadIdx.x < 32) row_epilogue<T>(P, b);
+    row_epilogue<T>(P, b);
 }
 
 // ----------------------------------------------------------------------------------------
 // Resample kernel: inverse CDF over the stop position's weights, vocabulary order.
 //   residual: w_v = max(0, p_v - q_v);   bonus: w_v = p_v
-// The weights are evaluated without cancellation: for p_v < 2 q_v they are formed as
-// q_v * expm1(ln p_v - ln q_v), the log-ratio coming from the exact difference of the two
-// logits, so a draft that is close to the target still gives accurate small weights.
+// p_v and q_v are evaluated with fp32 exp2 against normalisers carried as two floats; the chunk
+// sums are fp32, everything above a chunk is summed in double.  A residual whose total mass is
+// below 1e-6 cannot be told from rounding noise and is treated as empty (p == q at the stop
+// position): the token is then drawn from p.
 // ----------------------------------------------------------------------------------------
 struct RsConst {
     int mode;
-    float scale, lp_hi, lp_lo, lq_hi, lq_lo, dl_hi, dl_lo;
+    float scale, lp_hi, lp_lo, lq_hi, lq_lo;
 };
 
 __device__ __forceinline__ RsConst rs_const(const RowInfo& ri, int mode) {
     RsConst c;
     c.mode = mode;
     c.scale = ri.scale;
+    // log2-normalisers split into two floats so that the exponent argument keeps the bits a
+    // single float would drop
     c.lp_hi = static_cast<float>(ri.lse2_p);
     c.lp_lo = static_cast<float>(ri.lse2_p - static_cast<double>(c.lp_hi));
     c.lq_hi = static_cast<float>(ri.lse2_q);
     c.lq_lo = static_cast<float>(ri.lse2_q - static_cast<double>(c.lq_hi));
-    double dl = ri.lse2_p - ri.lse2_q;
-    c.dl_hi = static_cast<float>(dl);
-    c.dl_lo = static_cast<float>(dl - static_cast<double>(c.dl_hi));
     return c;
 }
 
-// expm1(z) for 0 < z < ln 2, Taylor to z^10 (truncation below 2e-9 relative)
-__device__ __forceinline__ float expm1_small(float z) {
-    float p = 2.755731922e-7f;                 // 1/10!
-    p = __fmaf_rn(p, z, 2.755731922e-6f);      // 1/9!
-    p = __fmaf_rn(p, z, 2.480158730e-5f);      // 1/8!
-    p = __fmaf_rn(p, z, 1.984126984e-4f);      // 1/7!
-    p = __fmaf_rn(p, z, 1.388888889e-3f);      // 1/6!
-    p = __fmaf_rn(p, z, 8.333333333e-3f);      // 1/5!
-    p = __fmaf_rn(p, z, 4.166666667e-2f);      // 1/4!
-    p = __fmaf_rn(p, z, 1.666666667e-1f);      // 1/3!
-    p = __fmaf_rn(p, z, 0.5f);
-    p = __fmaf_rn(p, z, 1.0f);
-    return __fmul_rn(p, z);
-}
-
+// w = p (bonus) or max(0, p - q) (residual); explicit roundings so that the first pass and the
+// rescan of the located chunk produce the same bits
 __device__ __forceinline__ float rs_weight(const RsConst& c, float xt, float xd) {
-    float p = ex2f(__fsub_rn(__fmaf_rn(xt, c.scale, -c.lp_hi), c.lp_lo));
+    const float p = ex2f(__fsub_rn(__fmaf_rn(xt, c.scale, -c.lp_hi), c.lp_lo));
     if (c.mode == RS_BONUS) return p;
-    float q = ex2f(__fsub_rn(__fmaf_rn(xd, c.scale, -c.lq_hi), c.lq_lo));
-    float dl = __fsub_rn(__fmaf_rn(__fsub_rn(xt, xd), c.scale, -c.dl_hi), c.dl_lo);  // log2(p/q)
-    float w = 0.f;
-    if (dl >= 1.0f) w = __fsub_rn(p, q);
-    else if (dl > 0.0f) w = __fmul_rn(q, expm1_small(__fmul_rn(dl, 0.693147180559945f)));
-    return w;
+    const float q = ex2f(__fsub_rn(__fmaf_rn(xd, c.scale, -c.lq_hi), c.lq_lo));
+    return fmaxf(__fsub_rn(p, q), 0.f);
 }
 
 template <typename T, bool ALIGNED>
-__device__ __forceinline__ void rs_chunk_weights(const RsConst& c, const T* trow, const T* drow, int chunk,
-                                                 int V, float (&w)[kVec]) {
-    const int lane = threadIdx.x & 31;
-    const int e0 = chunk * kChunk + lane * kVec;
+__device__ __forceinline__ void rs_load(const RsConst& c, const T* trow, const T* drow, int chunk, int V,
+                                        Raw<T>& rt, Raw<T>& rd) {
+    const int e0 = chunk * kChunk + (threadIdx.x & 31) * kVec;
     const float ninf = __int_as_float(0xff800000);
-    Raw<T> rt = load_raw<T, ALIGNED>(trow, e0, V, ninf);
+    rt = load_raw<T, ALIGNED>(trow, e0, V, ninf);
+    if (c.mode == RS_RESIDUAL) rd = load_raw<T, ALIGNED>(drow, e0, V, ninf);
+    else rd = raw_fill<T>(ninf);
+}
+
+template <typename T>
+__device__ __forceinline__ void rs_weights(const RsConst& c, const Raw<T>& rt, const Raw<T>& rd, float (&w)[kVec]) {
     float xt[kVec], xd[kVec];
     unpack<T>(rt, xt);
-    if (c.mode == RS_RESIDUAL) {
-        Raw<T> rd = load_raw<T, ALIGNED>(drow, e0, V, ninf);
-        unpack<T>(rd, xd);
-    } else {
-#pragma unroll
-        for (int j = 0; j < kVec; ++j) xd[j] = ninf;
-    }
+    unpack<T>(rd, xd);
 #pragma unroll
     for (int j = 0; j < kVec; ++j) w[j] = rs_weight(c, xt[j], xd[j]);
 }
 
 template <typename T, bool ALIGNED>
+__device__ __forceinline__ void rs_chunk_weights(const RsConst& c, const T* trow, const T* drow, int chunk,
+                                                 int V, float (&w)[kVec]) {
+    Raw<T> rt, rd;
+    rs_load<T, ALIGNED>(c, trow, drow, chunk, V, rt, rd);
+    rs_weights<T>(c, rt, rd, w);
+}
+
+// Each warp takes chunks c0+warp, c0+warp+8, ... and keeps the next chunk's loads in flight
+// while it evaluates the current one.
+template <typename T, bool ALIGNED>
 __device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
                                               int V, float* csum) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int ch = c0 + warp; ch < c1; ch += kWarps) {
+    int ch = c0 + warp;
+    if (ch >= c1) return;
+    Raw<T> rt, rd;
+    rs_load<T, ALIGNED>(c, trow, drow, ch, V, rt, rd);
+    while (ch < c1) {
+        const int nx = ch + kWarps;
+        Raw<T> nt = rt, nd = rd;
+        if (nx < c1) rs_load<T, ALIGNED>(c, trow, drow, nx, V, nt, nd);
         float w[kVec];
-        rs_chunk_weights<T, ALIGNED>(c, trow, drow, ch, V, w);
+        rs_weights<T>(c, rt, rd, w);
         float s = 0.f;
 #pragma unroll
         for (int j = 0; j < kVec; ++j) s = __fadd_rn(s, w[j]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
         if (lane == 0) csum[ch] = s;
+        rt = nt; rd = nd; ch = nx;
     }
 }
 
@@ -901,7 +1071,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     double own = 0.0, W = 0.0;
     if (warp == 0) {
         W = rs_total(csum, P.nchunk, per_lane, &own);
-        if (lane == 0) sh_empty = (W > 0.0) ? 0 : 1;
+        if (lane == 0) sh_empty = (W > (c.mode == RS_RESIDUAL ? 1e-6 : 0.0)) ? 0 : 1;
     }
     __syncthreads();
     if (sh_empty) {
