@@ -332,10 +332,6 @@ struct DraftState {
 
     template <typename T>
     __device__ __forceinline__ void step(Raw<T> raw, float scale) {
-#ifdef SPECKV_EXPERIMENT_NOMATH  // measurement only: keeps the loads, drops the arithmetic
-        cnt += __uint_as_float((raw.a.x ^ raw.a.y ^ raw.a.z ^ raw.a.w) & 0x007fffffu);
-        return;
-#endif
         if (raw_exceeds<false>(raw, m)) {  // an element >= m, or a NaN: rare after the warm start
             slow<T>(raw, scale);
             return;
@@ -399,10 +395,6 @@ struct TargetState {
     }
     template <typename T>
     __device__ __forceinline__ void step(const Raw<T>& raw, float scale) {
-#ifdef SPECKV_EXPERIMENT_NOMATH
-        r += __uint_as_float((raw.a.x ^ raw.a.y ^ raw.a.z ^ raw.a.w) & 0x007fffffu);
-        return;
-#endif
         if (raw_exceeds<true>(raw, m)) {  // a new maximum (or NaN): move the reference
             float vmax = raw_max(raw);
             if (vmax == vmax) {  // NaN needs no rescale; it poisons Z below
