@@ -49,7 +49,8 @@ typedef enum {
     SPECKV_ERR_INVALID_ARG = 1,
     SPECKV_ERR_UNSUPPORTED = 2,
     SPECKV_ERR_WORKSPACE = 3,
-    SPECKV_ERR_CUDA = 4
+    SPECKV_ERR_CUDA = 4,
+    SPECKV_ERR_STATIC_LIMIT = 5 /* batch needs more scratch than the built-in array holds */
 } speckv_status;
 
 typedef enum { SPECKV_F32 = 0, SPECKV_BF16 = 1 } speckv_dtype;
@@ -142,6 +143,33 @@ speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp,
                                    int32_t* row_status, void* workspace, size_t workspace_bytes,
                                    void* cuda_stream, void* ev_before_sweep, void* ev_after_sweep,
                                    void* ev_after_resample);
+
+/* speckv_signals for callers that cannot allocate device memory.  (The paper has no counterpart:
+ * this entry point exists for deployment reasons only.)
+ *
+ * Some hosts of this library may not call cudaMalloc once they are running: an inference server
+ * whose framework has already claimed all device memory for its own pool, a plug-in that is only
+ * allowed to touch buffers handed to it, a latency-critical decode loop where an allocation's
+ * implicit device synchronisation would stall every stream.  Such a caller has nowhere to get
+ * the workspace that speckv_signals asks for.  This variant brings its own: a fixed array of
+ * SPECKV_STATIC_SCRATCH_BYTES that is part of the library image, so every GPU that loads the
+ * library holds that much memory until the process exits.  The caller still owns and passes the
+ * inputs and the outputs; arguments, results and row_status are exactly those of speckv_signals.
+ *
+ *   - A batch whose speckv_workspace_size() exceeds SPECKV_STATIC_SCRATCH_BYTES is refused with
+ *     SPECKV_ERR_STATIC_LIMIT before anything is enqueued (B = 256, gamma_max = 8, V = 128256
+ *     needs 2.7 MB).
+ *   - The call allocates and frees nothing.  The first call on each device looks up the
+ *     array's device address (cudaGetSymbolAddress with that device current) and remembers it;
+ *     make that first call outside any stream capture.
+ *   - All calls on one device share the one array.  The parts that must start from zero are
+ *     cleared on the caller's stream at the start of each call; the rest keeps whatever the
+ *     previous call left.  Two calls that can overlap on the GPU (different streams without an
+ *     ordering between them) race on it: order them, or use speckv_signals with separate
+ *     workspaces.                                                                             */
+#define SPECKV_STATIC_SCRATCH_BYTES (4u << 20)
+speckv_status speckv_signals_static(const speckv_batch* batch, float* H, float* C, float* feat,
+                                    int32_t* row_status, void* cuda_stream);
 
 const char* speckv_status_string(speckv_status s);
 int speckv_version(void);

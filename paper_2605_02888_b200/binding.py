@@ -16,11 +16,12 @@ import torch
 
 from . import build as _build
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = range(5)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_STATIC_LIMIT = range(6)
 F32, BF16 = 0, 1
 ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE, ROW_TIMEOUT = 0, 1, 2, 4, 8, 16
 
-EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_select_gamma", "speckv_verify",
+STATIC_SCRATCH_BYTES = 4 << 20
+EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_signals_static", "speckv_select_gamma", "speckv_verify",
            "speckv_step", "speckv_step_profiled", "speckv_status_string", "speckv_version")
 
 
@@ -68,6 +69,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_workspace_size.argtypes = [C.POINTER(_CBatch), C.POINTER(sz)]
     L.speckv_signals.restype = C.c_int
     L.speckv_signals.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, vp, sz, vp]
+    L.speckv_signals_static.restype = C.c_int
+    L.speckv_signals_static.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, vp]
     L.speckv_select_gamma.restype = C.c_int
     L.speckv_select_gamma.argtypes = [C.c_int32, vp, vp, C.POINTER(_CMlp), vp, vp, vp]
     L.speckv_verify.restype = C.c_int
@@ -260,6 +263,24 @@ def speckv_signals(batch: Batch, out: Optional[StepOutputs] = None):
     if rc != OK:
         raise SpeckvError(rc, "speckv_signals")
     return dict(H=o.H, C=o.C, feat=o.feat, row_status=o.row_status)
+
+
+def speckv_signals_static(batch: Batch, H: torch.Tensor, Cc: torch.Tensor, feat: torch.Tensor,
+                          row_status: torch.Tensor):
+    """speckv_signals without a workspace argument, for callers that may not allocate device
+    memory: the scratch is a fixed array inside the library (STATIC_SCRATCH_BYTES per device).
+    All four outputs are caller-provided CUDA tensors; nothing is allocated here either.
+    Raises SpeckvError(ERR_STATIC_LIMIT) when the batch needs more scratch than that."""
+    L = load_library()
+    c = batch._c()
+    dev = batch.draft_logits.device
+    with torch.cuda.device(dev):
+        rc = L.speckv_signals_static(C.byref(c), _dev_ptr(H, torch.float32, "H"), _dev_ptr(Cc, torch.float32, "C"),
+                                     _dev_ptr(feat, torch.float32, "feat"),
+                                     _dev_ptr(row_status, torch.int32, "row_status"), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_signals_static")
+    return dict(H=H, C=Cc, feat=feat, row_status=row_status)
 
 
 def speckv_select_gamma(feat: torch.Tensor, comp: Optional[torch.Tensor], mlp: Mlp,

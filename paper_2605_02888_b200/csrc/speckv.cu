@@ -188,6 +188,25 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 
+// Scratch for speckv_signals_static: lives in the library image, one copy per device that loads it.
+static __device__ __align__(256) unsigned char g_static_scratch[SPECKV_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device.  In host code the array's name only
+// stands for the symbol; the address a kernel can use has to be asked for, once per device.
+cudaError_t static_scratch_address(void** out) {
+    static void* cached[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && cached[dev]) { *out = cached[dev]; return cudaSuccess; }
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) cached[dev] = p;
+    *out = p;
+    return cudaSuccess;
+}
+
 }  // namespace
 
 extern "C" {
@@ -206,6 +225,19 @@ speckv_status speckv_signals(const speckv_batch* batch, float* H, float* C, floa
                              void* cuda_stream) {
     return run(batch, MODE_SIGNALS, nullptr, nullptr, H, C, feat, nullptr, nullptr, nullptr, nullptr,
                row_status, workspace, workspace_bytes, cuda_stream);
+}
+
+speckv_status speckv_signals_static(const speckv_batch* batch, float* H, float* C, float* feat,
+                                    int32_t* row_status, void* cuda_stream) {
+    speckv_status st = check_batch(batch, false);
+    if (st != SPECKV_OK) return st;
+    if (batch->B == 0) return SPECKV_OK;
+    if (make_plan(batch).total > SPECKV_STATIC_SCRATCH_BYTES) return SPECKV_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    if (static_scratch_address(&scratch) != cudaSuccess || !scratch) return SPECKV_ERR_CUDA;
+    // run() clears the ticket counters on the caller's stream; nothing else needs a known start
+    return run(batch, MODE_SIGNALS, nullptr, nullptr, H, C, feat, nullptr, nullptr, nullptr, nullptr,
+               row_status, scratch, SPECKV_STATIC_SCRATCH_BYTES, cuda_stream);
 }
 
 speckv_status speckv_select_gamma(int32_t B, const float* feat, const float* comp,
@@ -261,6 +293,7 @@ const char* speckv_status_string(speckv_status s) {
         case SPECKV_ERR_UNSUPPORTED: return "unsupported size or type";
         case SPECKV_ERR_WORKSPACE: return "workspace too small";
         case SPECKV_ERR_CUDA: return "CUDA launch failed";
+        case SPECKV_ERR_STATIC_LIMIT: return "batch needs more scratch than the built-in array holds";
     }
     return "unknown status";
 }
