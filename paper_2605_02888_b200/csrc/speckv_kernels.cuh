@@ -58,6 +58,7 @@ struct RowInfo {  // written by the sweep kernel's row epilogue, read by the res
 
 struct KParams {
     int B, G, V, J, nsplit, nvec, per_split, nchunk, R, chunks_per_cta, mode, bits;
+    int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
     const void* t; long long tsb, tsp;
     const int* tok; const int* gamma; const float* temp; float temp_scalar; const float* u;
@@ -70,6 +71,7 @@ struct KParams {
     int *gamma_next, *n_acc, *out_tok, *status;
     // workspace
     int *tick1, *tick2;
+    int *qcount, *qhead, *qtail, *rowq;  // staged sweep: next quantum to hand out; queue of completed batch rows
     RowInfo* info;
     float4* part;
     float* csum;
@@ -639,133 +641,186 @@ __device__ __forceinline__ double warp_min(double v) {
     return v;
 }
 
-// Controller (Sec. 4.3, Eq. 1) for one row, executed by a full warp.  f4 = Hbar, cbar, Hmax, cmin.
-__device__ __forceinline__ void controller_row(const KParams& P, int b, const double (&f4)[4],
-                                               float* scores_row, int* gamma_next) {
+// Controller (Sec. 4.3, Eq. 1) for one row, executed by a full warp.  The parameters are fetched
+// first, all at once (ctl_load), so that their memory latency overlaps whatever comes between
+// the load and the evaluation.  Lane k holds hidden unit k's weights, b2[k] and comp[k].
+struct CtlRegs {
+    float w1[8], w2[8];
+    float b1, b2k, compk;
+};
+__device__ __forceinline__ CtlRegs ctl_load(const KParams& P, int b, int lane) {
+    CtlRegs c;
+    const bool hid = lane < P.n_hidden;
+#pragma unroll
+    for (int f = 0; f < 8; ++f) c.w1[f] = (hid && f < P.n_in) ? __ldg(P.W1 + lane * P.n_in + f) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) c.w2[j] = (hid && j < P.n_out) ? __ldg(P.W2 + j * P.n_hidden + lane) : 0.f;
+    c.b1 = hid ? __ldg(P.b1 + lane) : 0.f;
+    c.b2k = lane < P.n_out ? __ldg(P.b2 + lane) : 0.f;
+    c.compk = (P.comp && lane < P.n_comp) ? __ldg(P.comp + static_cast<long long>(b) * P.n_comp + lane) : 0.f;
+    return c;
+}
+// f4 = Hbar, cbar, Hmax, cmin
+__device__ __forceinline__ void ctl_eval(const KParams& P, const CtlRegs& c, const double (&f4)[4],
+                                         float* scores_row, int* gamma_next) {
     const int lane = threadIdx.x & 31;
     double x[8];
+    const int first_comp = (P.layout == 0) ? 3 : 4;
+    if (P.layout == 0) { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[3]; x[3] = 0.0; }
+    else { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[2]; x[3] = f4[3]; }
 #pragma unroll
-    for (int k = 0; k < 8; ++k) x[k] = 0.0;
-    const float* comp = P.comp ? P.comp + static_cast<long long>(b) * P.n_comp : nullptr;
-    if (P.layout == 0) {
-        x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[3];
-        for (int k = 3; k < P.n_in; ++k) x[k] = comp ? static_cast<double>(comp[k - 3]) : 0.0;
-    } else {
-        x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[2]; x[3] = f4[3];
-        for (int k = 4; k < P.n_in; ++k) x[k] = comp ? static_cast<double>(comp[k - 4]) : 0.0;
+    for (int k = 3; k < 8; ++k) {
+        const float cv = __shfl_sync(0xffffffffu, c.compk, (k - first_comp) & 31);
+        if (k >= first_comp) x[k] = (k < P.n_in) ? static_cast<double>(cv) : 0.0;
     }
-    double h = 0.0;
-    if (lane < P.n_hidden) {
-        h = static_cast<double>(P.b1[lane]);
-        for (int f = 0; f < P.n_in; ++f) h += static_cast<double>(P.W1[lane * P.n_in + f]) * x[f];
-        h = h > 0.0 ? h : 0.0;
-    }
+    double h = static_cast<double>(c.b1);
+#pragma unroll
+    for (int f = 0; f < 8; ++f)
+        if (f < P.n_in) h += static_cast<double>(c.w1[f]) * x[f];
+    h = (lane < P.n_hidden && h > 0.0) ? h : 0.0;
     double best = 0.0;
     int best_j = 0;
-    for (int j = 0; j < P.n_out; ++j) {
-        double part = (lane < P.n_hidden) ? static_cast<double>(P.W2[j * P.n_hidden + lane]) * h : 0.0;
-        double o = warp_sum(part) + static_cast<double>(P.b2[j]);
-        double e = (P.transform == 0) ? o * P.gch[j] + 1.0 : o;
-        if (scores_row && lane == 0) scores_row[j] = static_cast<float>(e);
-        if (j == 0 || e > best) { best = e; best_j = j; }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const double b2 = static_cast<double>(__shfl_sync(0xffffffffu, c.b2k, j));
+        if (j < P.n_out) {  // uniform across the warp
+            const double o = warp_sum(static_cast<double>(c.w2[j]) * h) + b2;
+            const double e = (P.transform == 0) ? o * P.gch[j] + 1.0 : o;
+            if (scores_row && lane == 0) scores_row[j] = static_cast<float>(e);
+            if (j == 0 || e > best) { best = e; best_j = j; }
+        }
     }
     if (gamma_next && lane == 0) *gamma_next = P.gch[best_j];
 }
 
-// Row epilogue: runs in warp 0 of the last CTA of batch row b.
+// Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
+// merges the nd partials at pd (draft position i) and the nt partials at pt (target position i).
+// gam and Tf are the row's gamma and temperature as the sweep read them.  Everything the row
+// needs from memory that does not depend on other loads is requested first, so the epilogue
+// costs two memory round trips (the second for the logits at the draft tokens).
 template <typename T>
-__device__ __noinline__ void row_epilogue(const KParams& P, int b) {
+__device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd, int nd,
+                                          const float4* pt, int nt) {
     const int lane = threadIdx.x & 31;
     const int G = P.G;
     const bool verify = (P.mode & MODE_VERIFY) != 0;
+    constexpr int kPre = 4;  // partials fetched ahead per lane; more are rare
 
-    int gam = P.gamma ? P.gamma[b] : G;
-    float Tf = P.temp ? P.temp[b] : P.temp_scalar;
     int status = 0;
     if (gam < 1 || gam > G) status |= 1;
     if (!(Tf >= 0.f) || Tf == __int_as_float(0x7f800000)) status |= 8;
     const bool greedy = (Tf == 0.f);
     const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
     const double sd = static_cast<double>(scale);
+    const bool dr_on = !status && lane < gam;
+    const bool tg_on = !status && verify && lane <= gam;
+    const bool tok_on = !status && verify && lane < gam;
 
+    // ---- first round trip ----
+    float4 qd[kPre], qt[kPre];
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) {
+        qd[k] = (dr_on && k < nd) ? ldcg4(pd + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+        qt[k] = (tg_on && k < nt) ? ldcg4(pt + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const long long urow = (static_cast<long long>(b) * (G + 1) + lane) * 2;
+    const int x = tok_on ? __ldg(P.tok + static_cast<long long>(b) * G + lane) : -1;
+    const float u_acc = tok_on ? __ldg(P.u + urow) : 0.f;
+    const float u_res = tg_on ? __ldg(P.u + urow + 1) : 0.f;
+    CtlRegs ctl;
+    if ((P.mode & MODE_MLP) && !status) ctl = ctl_load(P, b, lane);
+
+    // ---- second round trip: the two logits at the draft token ----
     const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb;
     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb;
+    const bool badtok = tok_on && (x < 0 || x >= P.V);
+    float dxf = 0.f, txf = 0.f;
+    if (tok_on && !badtok && !greedy) {
+        dxf = elem_to_float(drow + static_cast<long long>(lane) * P.dsp, x);
+        txf = elem_to_float(trow + static_cast<long long>(lane) * P.tsp, x);
+    }
 
     double Hi = 0.0, ci = 0.0, lse2_q = 0.0, lse2_p = 0.0;
     int amax = -1;
-    bool nonfinite = false, badtok = false, accept = true;
+    bool nonfinite = false, accept = true;
 
     if (!status) {
-        const bool dr_on = lane < gam;
-        const bool tg_on = verify && lane <= gam;
+        // The draft and the target merge below are written without branches (selects only) and do
+        // not depend on each other, so their instructions interleave; the scale factors between
+        // partials come from the fast fp32 exp2, the sums are carried in double.
+        // ---- draft: (m, cnt, Zx, S) partials, see merge_draft
+        double m = qd[0].x, cnt = qd[0].y, Zx = qd[0].z, S = qd[0].w;
+        {
+            auto fold = [&](const float4& q) {
+                const double qm = q.x, qc = q.y, qz = q.z, qs = q.w;
+                const double M = fmax(m, qm);
+                const double da = m - M, db = qm - M;
+                const double fa = static_cast<double>(ex2f(static_cast<float>(da * sd)));
+                const double fb = static_cast<double>(ex2f(static_cast<float>(db * sd)));
+                const double za = cnt + Zx, zb = qc + qz;
+                const bool ka = (m == M), kb = (qm == M);
+                const double ncnt = (ka ? cnt : 0.0) + (kb ? qc : 0.0);
+                Zx = (ka ? Zx : za * fa) + (kb ? qz : zb * fb);
+                S = (ka ? S : (S + da * za) * fa) + (kb ? qs : (qs + db * zb) * fb);
+                cnt = (cnt != cnt || qc != qc) ? __longlong_as_double(0x7ff8000000000000LL) : ncnt;
+                m = M;
+            };
+#pragma unroll
+            for (int k = 1; k < kPre; ++k)
+                if (k < nd) fold(qd[k]);
+            for (int k = kPre; k < nd; ++k) fold(ldcg4(pd + k));
+        }
+        // ---- target: (r, Z) partials, or (best, index, bad) for greedy rows
+        double R = qt[0].x, Zp = qt[0].y;
+        float bv = qt[0].x, bad = qt[0].z;
+        int bi = __float_as_int(qt[0].y);
+        {
+            auto fold = [&](const float4& q) {
+                const double qr = q.x;
+                const double Rn = fmax(R, qr);
+                Zp = Zp * static_cast<double>(ex2f(static_cast<float>(R - Rn))) +
+                     static_cast<double>(q.y) * static_cast<double>(ex2f(static_cast<float>(qr - Rn)));
+                R = Rn;
+                const int qi = __float_as_int(q.y);
+                const bool take = q.x > bv || (q.x == bv && qi < bi);
+                bv = take ? q.x : bv;
+                bi = take ? qi : bi;
+                bad += q.z;
+            };
+#pragma unroll
+            for (int k = 1; k < kPre; ++k)
+                if (k < nt) fold(qt[k]);
+            for (int k = kPre; k < nt; ++k) fold(ldcg4(pt + k));
+        }
         if (dr_on) {
-            const int j = verify ? (G + 1 + lane) : lane;
-            const float4* pp = P.part + (static_cast<long long>(b) * P.J + j) * P.nsplit;
-            double m = 0, cnt = 0, Zx = 0, S = 0;
-            for (int k = 0; k < P.nsplit; ++k) {
-                float4 q = ldcg4(pp + k);
-                double qm = q.x, qc = q.y, qz = q.z, qs = q.w;
-                if (k == 0) { m = qm; cnt = qc; Zx = qz; S = qs; continue; }
-                if (qm > m) {
-                    double dm = m - qm, f = exp2(dm * sd), za = cnt + Zx;
-                    Zx = za * f + qz; S = (S + dm * za) * f + qs; cnt = qc; m = qm;
-                } else if (qm == m) {
-                    cnt += qc; Zx += qz; S += qs;
-                } else {
-                    double dm = qm - m, f = exp2(dm * sd), za = qc + qz;
-                    Zx += za * f; S += (qs + dm * za) * f;
-                    if (qc != qc) cnt = qc;
-                }
-            }
-            double Z = cnt + Zx;
+            const double Z = cnt + Zx;
             if (!(cnt >= 1.0) || !(Z < 1e300) || !(m > static_cast<double>(kFloor))) {
                 nonfinite = true;
             } else {
-                double lnZ = log(cnt) + log1p(Zx / cnt);
-                Hi = lnZ - kLn2 * sd * S / Z;
+                const double lnZ = (cnt == 1.0) ? log1p(Zx) : log(cnt) + log1p(Zx / cnt);
+                const double rZ = 1.0 / Z;
+                Hi = lnZ - kLn2 * sd * S * rZ;
                 if (Hi < 0.0) Hi = 0.0;
-                ci = 1.0 / Z;
+                ci = rZ;
                 lse2_q = m * sd + lnZ * kLog2e;
             }
         }
         if (tg_on) {
-            const float4* pp = P.part + (static_cast<long long>(b) * P.J + lane) * P.nsplit;
             if (greedy) {
-                float bv = 0.f; int bi = 0x7fffffff; float bad = 0.f;
-                for (int k = 0; k < P.nsplit; ++k) {
-                    float4 q = ldcg4(pp + k);
-                    int qi = __float_as_int(q.y);
-                    if (k == 0 || q.x > bv || (q.x == bv && qi < bi)) { bv = q.x; bi = qi; }
-                    bad += q.z;
-                }
                 if (bad != 0.f || bi == 0x7fffffff || !(bv > kFloor)) nonfinite = true;
                 amax = bi;
             } else {
-                double R = 0, Z = 0;
-                for (int k = 0; k < P.nsplit; ++k) {
-                    float4 q = ldcg4(pp + k);
-                    double qr = q.x, qz = q.y;
-                    if (k == 0) { R = qr; Z = qz; continue; }
-                    if (qr > R) { Z = Z * exp2(R - qr) + qz; R = qr; }
-                    else { Z += qz * exp2(qr - R); }
-                }
-                if (!(Z > 0.0) || !(Z < 1e300)) nonfinite = true;
-                else lse2_p = R + log2(Z);
+                if (!(Zp > 0.0) || !(Zp < 1e300)) nonfinite = true;
+                else lse2_p = R + log2(Zp);
             }
         }
-        if (verify && lane < gam) {
-            int x = P.tok[static_cast<long long>(b) * G + lane];
-            if (x < 0 || x >= P.V) {
-                badtok = true;
-            } else if (greedy) {
+        if (tok_on && !badtok) {
+            if (greedy) {
                 accept = (x == amax);
             } else if (!nonfinite) {
-                double dx = static_cast<double>(elem_to_float(drow + static_cast<long long>(lane) * P.dsp, x));
-                double tx = static_cast<double>(elem_to_float(trow + static_cast<long long>(lane) * P.tsp, x));
-                double lq = dx * sd - lse2_q;
-                double lp = tx * sd - lse2_p;
-                double u = static_cast<double>(P.u[(static_cast<long long>(b) * (G + 1) + lane) * 2]);
-                accept = (log2(u) + lq) < lp;  // u * q(x) < p(x)
+                const double lq = static_cast<double>(dxf) * sd - lse2_q;
+                const double lp = static_cast<double>(txf) * sd - lse2_p;
+                accept = (log2(static_cast<double>(u_acc)) + lq) < lp;  // u * q(x) < p(x)
             }
         }
         if (__any_sync(0xffffffffu, nonfinite)) status |= 4;
@@ -773,13 +828,13 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
     }
 
     // first rejected position
-    unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);
-    int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
+    const unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);
+    const int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
 
     // signals
     const double in_bits = P.bits ? kLog2e : 1.0;
-    double Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.0;
-    double Cout = (status == 0 && lane < gam) ? ci : 0.0;
+    const double Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.0;
+    const double Cout = (status == 0 && lane < gam) ? ci : 0.0;
     double f4[4] = {0, 0, 0, 0};
     if (status == 0) {
         f4[0] = warp_sum(Hout) / gam;
@@ -795,8 +850,8 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
 
     if (P.mode & MODE_MLP) {
         if (status == 0) {
-            controller_row(P, b, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr,
-                           P.gamma_next + b);
+            ctl_eval(P, ctl, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr,
+                     P.gamma_next + b);
         } else {
             if (P.scores && lane < P.n_out) P.scores[static_cast<long long>(b) * P.n_out + lane] = 0.f;
             if (lane == 0) P.gamma_next[b] = 0;
@@ -804,14 +859,15 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
     }
 
     if (verify) {
-        // fresh token: known here for greedy rows, drawn by the resample kernel otherwise
-        int amax_n = __shfl_sync(0xffffffffu, amax, n);
-        double lp_n = __shfl_sync(0xffffffffu, lse2_p, n);
-        double lq_n = __shfl_sync(0xffffffffu, lse2_q, n < gam ? n : 0);
+        // fresh token: known here for greedy rows, drawn by the resample step otherwise
+        const int amax_n = __shfl_sync(0xffffffffu, amax, n);
+        const double lp_n = __shfl_sync(0xffffffffu, lse2_p, n);
+        const double lq_n = __shfl_sync(0xffffffffu, lse2_q, n < gam ? n : 0);
+        const float u2_n = __shfl_sync(0xffffffffu, u_res, n);
         if (lane <= G) {
             int v = -1;
             if (status == 0) {
-                if (lane < n) v = P.tok[static_cast<long long>(b) * G + lane];
+                if (lane < n) v = x;
                 else if (lane == n && greedy) v = amax_n;
             }
             P.out_tok[static_cast<long long>(b) * (G + 1) + lane] = v;
@@ -821,7 +877,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b) {
             RowInfo ri;
             ri.mode = (status == 0 && !greedy) ? (n < gam ? RS_RESIDUAL : RS_BONUS) : RS_NONE;
             ri.n = n;
-            ri.u2 = (status == 0 && !greedy) ? P.u[(static_cast<long long>(b) * (G + 1) + n) * 2 + 1] : 0.f;
+            ri.u2 = (status == 0 && !greedy) ? u2_n : 0.f;
             ri.scale = scale;
             ri.lse2_p = lp_n;
             ri.lse2_q = lq_n;
@@ -927,7 +983,9 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
     }
     if (!__shfl_sync(0xffffffffu, last_row, 0)) return;
     __threadfence();
-    row_epilogue<T>(P, b);
+    const long long row0 = static_cast<long long>(b) * P.J;
+    row_epilogue<T>(P, b, gam, Tf, P.part + (row0 + (verify ? P.G + 1 + lane : lane)) * P.nsplit, P.nsplit,
+                    P.part + (row0 + lane) * P.nsplit, P.nsplit);
 }
 
 // ----------------------------------------------------------------------------------------
@@ -1152,8 +1210,8 @@ __global__ void __launch_bounds__(kThreads) select_gamma_kernel(const __grid_con
     double f4[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) f4[k] = static_cast<double>(feat_in[static_cast<long long>(b) * 4 + k]);
-    controller_row(P, b, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr,
-                   P.gamma_next + b);
+    const CtlRegs ctl = ctl_load(P, b, threadIdx.x & 31);
+    ctl_eval(P, ctl, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr, P.gamma_next + b);
 }
 
 }  // namespace speckv
