@@ -8,6 +8,7 @@
 #include <cstdint>
 
 #include "speckv_kernels.cuh"
+#include "speckv_pipeline.cuh"
 
 namespace {
 
@@ -59,7 +60,7 @@ Plan make_plan(const speckv_batch* bt) {
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
     size_t off = 0;
-    p.off_tick = off; off = align_up(off + 2 * B * sizeof(int));
+    p.off_tick = off; off = align_up(off + (3 * B + 4) * sizeof(int));  // tickets, counters, row queue
     p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
     p.off_part = off; off = align_up(off + B * p.J_full * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
@@ -112,13 +113,42 @@ struct Events {  // optional timing events around the two kernels
     cudaEvent_t before_sweep = nullptr, after_sweep = nullptr, after_resample = nullptr;
 };
 
+// Staged sweep: persistent CTAs, two per SM.  Needs 16-byte aligned rows whose byte length is a
+// multiple of 16, and a batch whose per-row tables fit in shared memory.
+template <typename T>
+cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
+    static bool configured[64] = {};
+    static int n_sm[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const size_t smem = (sizeof(PipeShared) + 127) / 128 * 128 + static_cast<size_t>(kStages) * kStageBytes;
+    const bool slot = dev >= 0 && dev < 64;
+    int sms = slot ? n_sm[dev] : 0;
+    if (!slot || !configured[dev]) {
+        e = cudaFuncSetAttribute(pipe_sweep_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        if (slot) { n_sm[dev] = sms; configured[dev] = true; }
+    }
+    pipe_sweep_kernel<T><<<2 * sms, kPipeThreads, smem, st>>>(P);
+    return cudaGetLastError();
+}
+
 template <typename T, bool ALIGNED>
-cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev) {
+cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev, bool staged) {
     constexpr int U = sizeof(T) == 2 ? SPECKV_U : (SPECKV_U + 1) / 2;
     const long long grid = static_cast<long long>(P.B) * P.J * P.nsplit;
     if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
-    sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    if (ALIGNED && staged) {
+        e = launch_pipe<T>(P, st);
+    } else {
+        sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);
+        e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return e;
     if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
     if (P.mode & MODE_VERIFY) {
@@ -166,6 +196,10 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     char* w = static_cast<char*>(ws);
     P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
     P.tick2 = P.tick1 + P.B;
+    P.qcount = P.tick1 + 2 * P.B;
+    P.qhead = P.qcount + 1;
+    P.qtail = P.qcount + 2;
+    P.rowq = P.qcount + 4;
     P.info = reinterpret_cast<RowInfo*>(w + pl.off_info);
     P.part = reinterpret_cast<float4*>(w + pl.off_part);
     P.csum = reinterpret_cast<float*>(w + pl.off_csum);
@@ -173,18 +207,23 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(P.tick1, 0, 2 * static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess)
+    if (cudaMemsetAsync(P.tick1, 0, (3 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
 
     const int es = esize(bt->dtype);
     bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
     if (verify) aligned = aligned && rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
 
+    // the staged sweep wants whole 16-byte granules per row and a batch its per-row tables can hold
+    const long long row_bytes = static_cast<long long>(P.V) * es;
+    const bool staged = aligned && row_bytes % 16 == 0 && P.B <= kPipeMaxB;
+    P.Lg = static_cast<int>(row_bytes / 16);
+    P.Lp = (P.Lg + kStageGran - 1) / kStageGran * kStageGran;
     cudaError_t e;
     if (bt->dtype == SPECKV_BF16)
-        e = aligned ? launch_all<__nv_bfloat16, true>(P, cs, ev) : launch_all<__nv_bfloat16, false>(P, cs, ev);
+        e = aligned ? launch_all<__nv_bfloat16, true>(P, cs, ev, staged) : launch_all<__nv_bfloat16, false>(P, cs, ev, false);
     else
-        e = aligned ? launch_all<float, true>(P, cs, ev) : launch_all<float, false>(P, cs, ev);
+        e = aligned ? launch_all<float, true>(P, cs, ev, staged) : launch_all<float, false>(P, cs, ev, false);
     return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 

@@ -131,8 +131,9 @@ def test_signals_verify_and_controller_entry_points_agree_with_step():
     ver = speckv.speckv_verify(bt)
     ctl = speckv.speckv_select_gamma(sig["feat"], s["comp"], gm)
     torch.cuda.synchronize()
+    # the entry points cut the logit stream differently, so floats agree to rounding, not bit for bit
     for k in ("H", "C", "feat"):
-        assert torch.equal(sig[k], st[k]), k
+        close(sig[k].cpu().numpy(), st[k].cpu().numpy(), k, rtol=2e-6, atol=1e-7)
     for k in ("n_accepted", "out_tokens"):
         assert torch.equal(ver[k], st[k]), k
     assert torch.equal(ctl["gamma_next"], st["gamma_next"])
