@@ -660,37 +660,45 @@ __device__ __forceinline__ CtlRegs ctl_load(const KParams& P, int b, int lane) {
     c.compk = (P.comp && lane < P.n_comp) ? __ldg(P.comp + static_cast<long long>(b) * P.n_comp + lane) : 0.f;
     return c;
 }
-// f4 = Hbar, cbar, Hmax, cmin
-__device__ __forceinline__ void ctl_eval(const KParams& P, const CtlRegs& c, const double (&f4)[4],
+// f4 = Hbar, cbar, Hmax, cmin.  fp32 throughout: 164 multiply-adds on values of order one.
+__device__ __forceinline__ void ctl_eval(const KParams& P, const CtlRegs& c, const float (&f4)[4],
                                          float* scores_row, int* gamma_next) {
     const int lane = threadIdx.x & 31;
-    double x[8];
+    float x[8];
     const int first_comp = (P.layout == 0) ? 3 : 4;
-    if (P.layout == 0) { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[3]; x[3] = 0.0; }
+    if (P.layout == 0) { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[3]; x[3] = 0.f; }
     else { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[2]; x[3] = f4[3]; }
 #pragma unroll
     for (int k = 3; k < 8; ++k) {
         const float cv = __shfl_sync(0xffffffffu, c.compk, (k - first_comp) & 31);
-        if (k >= first_comp) x[k] = (k < P.n_in) ? static_cast<double>(cv) : 0.0;
+        if (k >= first_comp) x[k] = (k < P.n_in) ? cv : 0.f;
     }
-    double h = static_cast<double>(c.b1);
+    float h = c.b1;
 #pragma unroll
     for (int f = 0; f < 8; ++f)
-        if (f < P.n_in) h += static_cast<double>(c.w1[f]) * x[f];
-    h = (lane < P.n_hidden && h > 0.0) ? h : 0.0;
-    double best = 0.0;
+        if (f < P.n_in) h = fmaf(c.w1[f], x[f], h);
+    h = (lane < P.n_hidden && h > 0.f) ? h : 0.f;
+    float best = 0.f;
     int best_j = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const double b2 = static_cast<double>(__shfl_sync(0xffffffffu, c.b2k, j));
+        const float b2 = __shfl_sync(0xffffffffu, c.b2k, j);
         if (j < P.n_out) {  // uniform across the warp
-            const double o = warp_sum(static_cast<double>(c.w2[j]) * h) + b2;
-            const double e = (P.transform == 0) ? o * P.gch[j] + 1.0 : o;
-            if (scores_row && lane == 0) scores_row[j] = static_cast<float>(e);
+            const float o = warp_sumf(c.w2[j] * h) + b2;
+            const float e = (P.transform == 0) ? fmaf(o, static_cast<float>(P.gch[j]), 1.f) : o;
+            if (scores_row && lane == 0) scores_row[j] = e;
             if (j == 0 || e > best) { best = e; best_j = j; }
         }
     }
     if (gamma_next && lane == 0) *gamma_next = P.gch[best_j];
+}
+
+// log2 of a positive finite number as an exact integer part plus the fp32 log2 of the mantissa
+// (below one in magnitude, so its absolute error stays near 1e-7 however large the argument)
+__device__ __forceinline__ double log2_split(double z) {
+    int k;
+    const double m = frexp(z, &k);  // m in [0.5, 1)
+    return static_cast<double>(k) + static_cast<double>(log2f(static_cast<float>(m)));
 }
 
 // Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
@@ -740,113 +748,67 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         txf = elem_to_float(trow + static_cast<long long>(lane) * P.tsp, x);
     }
 
-    double Hi = 0.0, ci = 0.0, lse2_q = 0.0, lse2_p = 0.0;
+    float Hi = 0.f, ci = 0.f;
+    double lse2_q = 0.0, lse2_p = 0.0;
     int amax = -1;
     bool nonfinite = false, accept = true;
 
     if (!status) {
-        // The draft and the target merge below are written without branches (selects only) and do
-        // not depend on each other, so their instructions interleave; the scale factors between
-        // partials come from the fast fp32 exp2, the sums are carried in double.
-        // ---- draft: (m, cnt, Zx, S) partials, see merge_draft
-        double m = qd[0].x, cnt = qd[0].y, Zx = qd[0].z, S = qd[0].w;
-        {
-            auto fold = [&](const float4& q) {
-                const double qm = q.x, qc = q.y, qz = q.z, qs = q.w;
-                const double M = fmax(m, qm);
-                const double da = m - M, db = qm - M;
-                const double fa = static_cast<double>(ex2f(static_cast<float>(da * sd)));
-                const double fb = static_cast<double>(ex2f(static_cast<float>(db * sd)));
-                const double za = cnt + Zx, zb = qc + qz;
-                const bool ka = (m == M), kb = (qm == M);
-                const double ncnt = (ka ? cnt : 0.0) + (kb ? qc : 0.0);
-                Zx = (ka ? Zx : za * fa) + (kb ? qz : zb * fb);
-                S = (ka ? S : (S + da * za) * fa) + (kb ? qs : (qs + db * zb) * fb);
-                cnt = (cnt != cnt || qc != qc) ? __longlong_as_double(0x7ff8000000000000LL) : ncnt;
-                m = M;
-            };
+        // Partials are merged in fp32 with the same branch-free rules the sweep uses; the draft and
+        // the target chain are independent, so their instructions interleave.  Only what decides an
+        // acceptance (the log2-normalisers and the test itself) is carried in double.
+        float4 ad = qd[0], at = qt[0];
 #pragma unroll
-            for (int k = 1; k < kPre; ++k)
-                if (k < nd) fold(qd[k]);
-            for (int k = kPre; k < nd; ++k) fold(ldcg4(pd + k));
+        for (int k = 1; k < kPre; ++k) {
+            if (k < nd) ad = merge_draft(ad, qd[k], scale);
+            if (k < nt) at = greedy ? merge_argmax(at, qt[k]) : merge_target(at, qt[k]);
         }
-        // ---- target: (r, Z) partials, or (best, index, bad) for greedy rows
-        double R = qt[0].x, Zp = qt[0].y;
-        float bv = qt[0].x, bad = qt[0].z;
-        int bi = __float_as_int(qt[0].y);
-        {
-            auto fold = [&](const float4& q) {
-                const double qr = q.x;
-                const double Rn = fmax(R, qr);
-                Zp = Zp * static_cast<double>(ex2f(static_cast<float>(R - Rn))) +
-                     static_cast<double>(q.y) * static_cast<double>(ex2f(static_cast<float>(qr - Rn)));
-                R = Rn;
-                const int qi = __float_as_int(q.y);
-                const bool take = q.x > bv || (q.x == bv && qi < bi);
-                bv = take ? q.x : bv;
-                bi = take ? qi : bi;
-                bad += q.z;
-            };
-#pragma unroll
-            for (int k = 1; k < kPre; ++k)
-                if (k < nt) fold(qt[k]);
-            for (int k = kPre; k < nt; ++k) fold(ldcg4(pt + k));
-        }
+        for (int k = kPre; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
+        for (int k = kPre; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
         if (dr_on) {
-            const double Z = cnt + Zx;
-            if (!(cnt >= 1.0) || !(Z < 1e300) || !(m > static_cast<double>(kFloor))) {
+            const float m = ad.x, cnt = ad.y, Zx = ad.z, S = ad.w;
+            const float Z = cnt + Zx;
+            if (!(cnt >= 1.f) || !(Z < 3e38f) || !(m > kFloor)) {
                 nonfinite = true;
             } else {
-                const double lnZ = (cnt == 1.0) ? log1p(Zx) : log(cnt) + log1p(Zx / cnt);
-                const double rZ = 1.0 / Z;
-                Hi = lnZ - kLn2 * sd * S * rZ;
-                if (Hi < 0.0) Hi = 0.0;
+                const float lnZ = (cnt == 1.f) ? log1pf(Zx) : logf(cnt) + log1pf(Zx / cnt);
+                const float rZ = 1.f / Z;
+                Hi = fmaxf(lnZ - static_cast<float>(kLn2) * scale * S * rZ, 0.f);
                 ci = rZ;
-                lse2_q = m * sd + lnZ * kLog2e;
+                lse2_q = static_cast<double>(m) * sd + log2_split(static_cast<double>(cnt) + static_cast<double>(Zx));
             }
         }
         if (tg_on) {
             if (greedy) {
-                if (bad != 0.f || bi == 0x7fffffff || !(bv > kFloor)) nonfinite = true;
+                const int bi = __float_as_int(at.y);
+                if (at.z != 0.f || bi == 0x7fffffff || !(at.x > kFloor)) nonfinite = true;
                 amax = bi;
             } else {
-                if (!(Zp > 0.0) || !(Zp < 1e300)) nonfinite = true;
-                else lse2_p = R + log2(Zp);
-            }
-        }
-        if (tok_on && !badtok) {
-            if (greedy) {
-                accept = (x == amax);
-            } else if (!nonfinite) {
-                const double lq = static_cast<double>(dxf) * sd - lse2_q;
-                const double lp = static_cast<double>(txf) * sd - lse2_p;
-                accept = (log2(static_cast<double>(u_acc)) + lq) < lp;  // u * q(x) < p(x)
+                if (!(at.y > 0.f) || !(at.y < 3e38f)) nonfinite = true;
+                else lse2_p = static_cast<double>(at.x) + log2_split(static_cast<double>(at.y));
             }
         }
         if (__any_sync(0xffffffffu, nonfinite)) status |= 4;
         if (__any_sync(0xffffffffu, badtok)) status |= 2;
     }
 
-    // first rejected position
-    const unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);
-    const int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
-
     // signals
-    const double in_bits = P.bits ? kLog2e : 1.0;
-    const double Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.0;
-    const double Cout = (status == 0 && lane < gam) ? ci : 0.0;
-    double f4[4] = {0, 0, 0, 0};
+    const float in_bits = P.bits ? static_cast<float>(kLog2e) : 1.f;
+    const float Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.f;
+    const float Cout = (status == 0 && lane < gam) ? ci : 0.f;
+    float f4[4] = {0.f, 0.f, 0.f, 0.f};
     if (status == 0) {
-        f4[0] = warp_sum(Hout) / gam;
-        f4[1] = warp_sum(Cout) / gam;
-        f4[2] = warp_max(Hout);
-        f4[3] = warp_min(lane < gam ? Cout : 2.0);
+        f4[0] = warp_sumf(Hout) / static_cast<float>(gam);
+        f4[1] = warp_sumf(Cout) / static_cast<float>(gam);
+        f4[2] = warp_maxf(Hout);
+        f4[3] = -warp_maxf(lane < gam ? -Cout : -2.f);
     }
     if (lane < G) {
-        if (P.H) P.H[static_cast<long long>(b) * G + lane] = static_cast<float>(Hout);
-        if (P.C) P.C[static_cast<long long>(b) * G + lane] = static_cast<float>(Cout);
+        if (P.H) P.H[static_cast<long long>(b) * G + lane] = Hout;
+        if (P.C) P.C[static_cast<long long>(b) * G + lane] = Cout;
     }
-    if (P.feat && lane < 4) P.feat[static_cast<long long>(b) * 4 + lane] = static_cast<float>(f4[lane]);
+    if (P.feat && lane < 4)
+        P.feat[static_cast<long long>(b) * 4 + lane] = lane == 0 ? f4[0] : lane == 1 ? f4[1] : lane == 2 ? f4[2] : f4[3];
 
     if (P.mode & MODE_MLP) {
         if (status == 0) {
@@ -857,6 +819,22 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             if (lane == 0) P.gamma_next[b] = 0;
         }
     }
+
+    // acceptance comes last: the two logits at the draft token had the whole signal and controller
+    // work above to arrive
+    if (status == 0 && tok_on) {
+        if (greedy) {
+            accept = (x == amax);
+        } else {
+            const double lq = static_cast<double>(dxf) * sd - lse2_q;
+            const double lp = static_cast<double>(txf) * sd - lse2_p;
+            // u * q(x) < p(x); u = 0 gives -inf on the left
+            const double l2u = (u_acc > 0.f) ? log2_split(static_cast<double>(u_acc)) : -__longlong_as_double(0x7ff0000000000000LL);
+            accept = (l2u + lq) < lp;
+        }
+    }
+    const unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);  // first rejected position
+    const int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
 
     if (verify) {
         // fresh token: known here for greedy rows, drawn by the resample step otherwise
@@ -1207,9 +1185,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
 __global__ void __launch_bounds__(kThreads) select_gamma_kernel(const __grid_constant__ KParams P, const float* feat_in) {
     const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
     if (b >= P.B) return;
-    double f4[4];
+    float f4[4];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) f4[k] = static_cast<double>(feat_in[static_cast<long long>(b) * 4 + k]);
+    for (int k = 0; k < 4; ++k) f4[k] = feat_in[static_cast<long long>(b) * 4 + k];
     const CtlRegs ctl = ctl_load(P, b, threadIdx.x & 31);
     ctl_eval(P, ctl, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr, P.gamma_next + b);
 }
