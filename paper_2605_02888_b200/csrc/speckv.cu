@@ -152,7 +152,7 @@ cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev, bool
     if (e != cudaSuccess) return e;
     if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
     if (P.mode & MODE_VERIFY) {
-        resample_kernel<T, ALIGNED><<<dim3(P.B, P.R), kThreads, 0, st>>>(P);
+        resample_kernel<T, ALIGNED><<<static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R), kThreads, 0, st>>>(P);
         e = cudaGetLastError();
     }
     if (ev.after_resample) cudaEventRecord(ev.after_resample, st);

@@ -1011,13 +1011,34 @@ __device__ __forceinline__ void rs_load(const RsConst& c, const T* trow, const T
     else rd = raw_fill<T>(ninf);
 }
 
+// the kVec weights of one lane, two elements per instruction; per element the same operations and
+// roundings as rs_weight, so both give the same bits
 template <typename T>
 __device__ __forceinline__ void rs_weights(const RsConst& c, const Raw<T>& rt, const Raw<T>& rd, float (&w)[kVec]) {
-    float xt[kVec], xd[kVec];
-    unpack<T>(rt, xt);
-    unpack<T>(rd, xd);
+    const f2 sc2 = pack2(c.scale, c.scale);
+    const f2 ph2 = pack2(-c.lp_hi, -c.lp_hi), pl2 = pack2(c.lp_lo, c.lp_lo);
+    f2 xt[4];
+    unpack_pairs(rt, xt);
+    if (c.mode == RS_BONUS) {
 #pragma unroll
-    for (int j = 0; j < kVec; ++j) w[j] = rs_weight(c, xt[j], xd[j]);
+        for (int i = 0; i < 4; ++i) {
+            const f2 p = ex2_2(sub2(fma2(xt[i], sc2, ph2), pl2));
+            unpack2(p, w[2 * i], w[2 * i + 1]);
+        }
+        return;
+    }
+    const f2 qh2 = pack2(-c.lq_hi, -c.lq_hi), ql2 = pack2(c.lq_lo, c.lq_lo);
+    f2 xd[4];
+    unpack_pairs(rd, xd);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const f2 p = ex2_2(sub2(fma2(xt[i], sc2, ph2), pl2));
+        const f2 q = ex2_2(sub2(fma2(xd[i], sc2, qh2), ql2));
+        float lo, hi;
+        unpack2(sub2(p, q), lo, hi);
+        w[2 * i] = fmaxf(lo, 0.f);
+        w[2 * i + 1] = fmaxf(hi, 0.f);
+    }
 }
 
 template <typename T, bool ALIGNED>
@@ -1028,38 +1049,85 @@ __device__ __forceinline__ void rs_chunk_weights(const RsConst& c, const T* trow
     rs_weights<T>(c, rt, rd, w);
 }
 
-// Each warp takes chunks c0+warp, c0+warp+8, ... and keeps the next chunk's loads in flight
-// while it evaluates the current one.
+// Each warp takes two chunks at a time (c0+warp, +8) and requests the next two before it evaluates
+// the current ones, so the memory latency is paid once per CTA, not once per batch.
 template <typename T, bool ALIGNED>
-__device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
-                                              int V, float* csum) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    int ch = c0 + warp;
-    if (ch >= c1) return;
-    Raw<T> rt, rd;
-    rs_load<T, ALIGNED>(c, trow, drow, ch, V, rt, rd);
-    while (ch < c1) {
-        const int nx = ch + kWarps;
-        Raw<T> nt = rt, nd = rd;
-        if (nx < c1) rs_load<T, ALIGNED>(c, trow, drow, nx, V, nt, nd);
-        float w[kVec];
-        rs_weights<T>(c, rt, rd, w);
-        float s = 0.f;
+__device__ __forceinline__ void rs_load_batch(const RsConst& c, const T* trow, const T* drow, int base, int c1, int V,
+                                              Raw<T> (&rt)[2], Raw<T> (&rd)[2]) {
 #pragma unroll
-        for (int j = 0; j < kVec; ++j) s = __fadd_rn(s, w[j]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s = __fadd_rn(s, __shfl_xor_sync(0xffffffffu, s, o));
-        if (lane == 0) csum[ch] = s;
-        rt = nt; rd = nd; ch = nx;
+    for (int u = 0; u < 2; ++u) {
+        const int ch = base + u * kWarps;
+        if (ch < c1) rs_load<T, ALIGNED>(c, trow, drow, ch, V, rt[u], rd[u]);
+        else { rt[u] = raw_fill<T>(__int_as_float(0xff800000)); rd[u] = rt[u]; }
     }
 }
 
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
+                                              int V, float* csum) {
+    constexpr int kU = 2;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    int base = c0 + warp;
+    if (base >= c1) return;
+    Raw<T> rt[kU], rd[kU];
+    rs_load_batch<T, ALIGNED>(c, trow, drow, base, c1, V, rt, rd);
+    while (base < c1) {
+        const int next = base + kWarps * kU;
+        Raw<T> nt[kU], nd[kU];
+        if (next < c1) rs_load_batch<T, ALIGNED>(c, trow, drow, next, c1, V, nt, nd);
+        float s[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            float w[kVec];
+            rs_weights<T>(c, rt[u], rd[u], w);
+            s[u] = 0.f;
+#pragma unroll
+            for (int j = 0; j < kVec; ++j) s[u] = __fadd_rn(s[u], w[j]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int u = 0; u < kU; ++u) s[u] = __fadd_rn(s[u], __shfl_xor_sync(0xffffffffu, s[u], o));
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int ch = base + u * kWarps;
+            if (lane == 0 && ch < c1) csum[ch] = s[u];
+        }
+        if (next < c1) {
+#pragma unroll
+            for (int u = 0; u < kU; ++u) { rt[u] = nt[u]; rd[u] = nd[u]; }
+        }
+        base = next;
+    }
+}
+
+// The last CTA of a row copies the row's chunk sums into shared memory (one memory round trip for
+// all of them) before it searches them; rows with more chunks than fit are searched in place.
+constexpr int kRsStage = 2048;
+struct RsSums {
+    const float* sh;    // staged copy, or nullptr
+    const float* glob;
+    __device__ __forceinline__ float operator[](int ch) const { return sh ? sh[ch] : __ldcg(glob + ch); }
+};
+__device__ __forceinline__ RsSums rs_stage_sums(float* sh_cs, const float* csum, int nchunk) {
+    RsSums r;
+    r.glob = csum;
+    r.sh = nullptr;
+    if (nchunk <= kRsStage) {
+        for (int ch = threadIdx.x; ch < nchunk; ch += kThreads) sh_cs[ch] = __ldcg(csum + ch);
+        r.sh = sh_cs;
+    }
+    __syncthreads();
+    return r;
+}
+
 // warp 0: total weight W of the row from its chunk sums
-__device__ __forceinline__ double rs_total(const float* csum, int nchunk, int per_lane, double* own_out) {
+__device__ __forceinline__ double rs_total(const RsSums& cs, int nchunk, int per_lane, double* own_out) {
     const int lane = threadIdx.x & 31;
     double own = 0.0;
     const int a = lane * per_lane, e = min(nchunk, a + per_lane);
-    for (int ch = a; ch < e; ++ch) own += static_cast<double>(__ldcg(csum + ch));
+    for (int ch = a; ch < e; ++ch) own += static_cast<double>(cs[ch]);
     *own_out = own;
     return warp_sum(own);
 }
@@ -1068,7 +1136,11 @@ template <typename T, bool ALIGNED>
 __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ KParams P) {
     __shared__ int sh_flag;
     __shared__ int sh_empty;
-    const int b = blockIdx.x;  // batch row; blockIdx.y = which share of the row's chunks
+    __shared__ float sh_cs[kRsStage];
+    // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
+    // launch order, so rows finish one after the other and their searches overlap the other rows' sums
+    const int b = blockIdx.x / P.R;
+    const int share = blockIdx.x - b * P.R;
     const RowInfo ri = P.info[b];
     if (ri.mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
 
@@ -1079,7 +1151,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     float* csum = P.csum + static_cast<long long>(b) * P.nchunk;
     RsConst c = rs_const(ri, ri.mode);
 
-    const int c0 = blockIdx.y * P.chunks_per_cta;
+    const int c0 = share * P.chunks_per_cta;
     const int c1 = min(P.nchunk, c0 + P.chunks_per_cta);
     rs_chunk_sums<T, ALIGNED>(c, trow, drow, c0, c1, P.V, csum);
 
@@ -1087,7 +1159,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     if (threadIdx.x == 0) {
         __threadfence();
         int old = atomicAdd(P.tick2 + b, 1);
-        sh_flag = (old == static_cast<int>(gridDim.y) - 1);
+        sh_flag = (old == P.R - 1);
     }
     __syncthreads();
     if (!sh_flag) return;
@@ -1097,8 +1169,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int per_lane = (P.nchunk + 31) / 32;
     double own = 0.0, W = 0.0;
+    RsSums cs = rs_stage_sums(sh_cs, csum, P.nchunk);
     if (warp == 0) {
-        W = rs_total(csum, P.nchunk, per_lane, &own);
+        W = rs_total(cs, P.nchunk, per_lane, &own);
         if (lane == 0) sh_empty = (W > (c.mode == RS_RESIDUAL ? 1e-6 : 0.0)) ? 0 : 1;
     }
     __syncthreads();
@@ -1111,7 +1184,8 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         c.mode = RS_BONUS;
         rs_chunk_sums<T, ALIGNED>(c, trow, drow, 0, P.nchunk, P.V, csum);
         __syncthreads();
-        if (warp == 0) W = rs_total(csum, P.nchunk, per_lane, &own);
+        cs = rs_stage_sums(sh_cs, csum, P.nchunk);
+        if (warp == 0) W = rs_total(cs, P.nchunk, per_lane, &own);
     }
     if (warp != 0) return;
 
@@ -1135,7 +1209,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         int last_pos = -1;
         double last_before = 0.0;
         for (int ch = a; ch < e; ++ch) {
-            double sv = static_cast<double>(__ldcg(csum + ch));
+            double sv = static_cast<double>(cs[ch]);
             if (sv > 0.0) { last_pos = ch; last_before = run; }
             if (run + sv > tau && sv > 0.0) { chunk = ch; before = run; break; }
             run += sv;
