@@ -133,7 +133,7 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         if (slot) { n_sm[dev] = sms; configured[dev] = true; }
     }
-    pipe_sweep_kernel<T><<<2 * sms, kPipeThreads, smem, st>>>(P);
+    pipe_sweep_kernel<T><<<SPECKV_PIPE_CTAS * sms, kPipeThreads, smem, st>>>(P);
     return cudaGetLastError();
 }
 
@@ -152,8 +152,19 @@ cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev, bool
     if (e != cudaSuccess) return e;
     if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
     if (P.mode & MODE_VERIFY) {
-        resample_kernel<T, ALIGNED><<<static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R), kThreads, 0, st>>>(P);
-        e = cudaGetLastError();
+        // programmatic dependent launch: the kernel's CTAs are scheduled while the sweep drains and
+        // wait inside the kernel for the sweep's results
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R));
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, resample_kernel<T, ALIGNED>, P);
     }
     if (ev.after_resample) cudaEventRecord(ev.after_resample, st);
     return e;
@@ -216,7 +227,15 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
 
     // the staged sweep wants whole 16-byte granules per row and a batch its per-row tables can hold
     const long long row_bytes = static_cast<long long>(P.V) * es;
-    const bool staged = aligned && row_bytes % 16 == 0 && P.B <= kPipeMaxB;
+    // Which sweep.  Measured on B200 (full-size workloads, same inputs): fp32 logits are bound by
+    // memory and the bulk-copy ring is faster (6.7-6.8 against 6.4 TB/s); bf16 logits need one
+    // exponential per two bytes and are bound by the special-function pipe, where the
+    // register-staged kernel with its 32 warps per SM hides latency better (4.95 against 4.6 TB/s).
+#ifndef SPECKV_STAGED
+#define SPECKV_STAGED 1  // 0: never, 1: fp32 only, 2: whenever the layout allows (measurement builds)
+#endif
+    const bool staged = (SPECKV_STAGED == 2 || (SPECKV_STAGED == 1 && bt->dtype == SPECKV_F32)) && aligned &&
+                        row_bytes % 16 == 0 && P.B <= kPipeMaxB;
     P.Lg = static_cast<int>(row_bytes / 16);
     P.Lp = (P.Lg + kStageGran - 1) / kStageGran * kStageGran;
     cudaError_t e;

@@ -873,6 +873,7 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
     __shared__ float4 sh_part[kWarps];
     __shared__ int sh_count;
     __shared__ float sh_m0[kWarps];
+    asm volatile("griddepcontrol.launch_dependents;");  // the resample kernel may be scheduled as SMs free up
     if (threadIdx.x == 0) sh_count = 0;
     if (threadIdx.x < kWarps) sh_m0[threadIdx.x] = kFloor;
     __syncthreads();  // before any load is issued
@@ -1137,6 +1138,9 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     __shared__ int sh_flag;
     __shared__ int sh_empty;
     __shared__ float sh_cs[kRsStage];
+    // launched as a programmatic dependent of the sweep kernel: its CTAs may already be resident
+    // while the sweep's last CTAs finish; nothing the sweep wrote is read before this returns
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
     const int b = blockIdx.x / P.R;

@@ -25,7 +25,10 @@
 
 namespace speckv {
 
-constexpr int kPipeWarps = 8;                        // consumer warps per CTA
+#ifndef SPECKV_PIPE_WARPS
+#define SPECKV_PIPE_WARPS 8
+#endif
+constexpr int kPipeWarps = SPECKV_PIPE_WARPS;        // consumer warps per CTA
 constexpr int kPipeThreads = (kPipeWarps + 2) * 32;  // + one producer warp + one epilogue warp
 #ifndef SPECKV_STAGE_GRAN
 #define SPECKV_STAGE_GRAN 1024                       // 16-byte granules per ring stage (16 KB)
@@ -34,13 +37,22 @@ constexpr int kPipeThreads = (kPipeWarps + 2) * 32;  // + one producer warp + on
 #define SPECKV_STAGES 6
 #endif
 #ifndef SPECKV_QUANTUM_STAGES
-#define SPECKV_QUANTUM_STAGES 8                      // target quantum: 128 KB
+#define SPECKV_QUANTUM_STAGES 16                     // target quantum: 256 KB
 #endif
 constexpr int kStageGran = SPECKV_STAGE_GRAN;
 constexpr int kStageBytes = kStageGran * 16;
 constexpr int kStages = SPECKV_STAGES;
-constexpr int kSegSlots = 32;                        // segments between the consumers and the epilogue warp
-constexpr int kPipeMaxB = 1024;                      // batch rows whose per-row tables fit the CTA
+#ifndef SPECKV_SEG_SLOTS
+#define SPECKV_SEG_SLOTS 32
+#endif
+#ifndef SPECKV_PIPE_MAXB
+#define SPECKV_PIPE_MAXB 1024
+#endif
+#ifndef SPECKV_PIPE_CTAS
+#define SPECKV_PIPE_CTAS 2                           // CTAs per SM
+#endif
+constexpr int kSegSlots = SPECKV_SEG_SLOTS;          // segments between the consumers and the epilogue warp
+constexpr int kPipeMaxB = SPECKV_PIPE_MAXB;          // batch rows whose per-row tables fit the CTA
 constexpr int kMaxSeg = 32;                          // partial slots per logit row
 constexpr int kWaitLimit = 1 << 22;
 
@@ -72,6 +84,7 @@ struct PipeShared {
     float4 part[kSegSlots][kPipeWarps];
     int error;
     int total_segs;                           // -1 until the producer has issued its last segment
+    int published;                            // set once the epilogue warp has published them all
     long long Q, Tg;                          // quantum and stream length, in granules
     int prefix[kPipeMaxB + 1];                // logit rows of the stream before each batch row
     float temp[kPipeMaxB];                    // the rows' temperature and gamma, read once
@@ -463,6 +476,26 @@ __device__ __forceinline__ void pipe_row_job(const KParams& P, PipeShared& sh, i
     row_epilogue<T>(P, b, gam, sh.temp[b], pd, nd, pt, nt);
 }
 
+// Take a completed batch row off the global queue (whole warp; the answer is the same in all lanes):
+// the row, or -1: queue empty, or -2: lost the claim to another warp, look again.
+__device__ __forceinline__ int pipe_pop_row(const KParams& P, volatile int* error, int lane) {
+    int b = -1;
+    if (lane == 0) {
+        const int h = ld_volatile(P.qhead);
+        if (h < ld_volatile(P.qtail)) {
+            b = -2;
+            if (atomicCAS(P.qhead, h, h + 1) == h) {
+                int v = 0;
+                for (int it = 0; it < kWaitLimit && v == 0; ++it) v = ld_volatile(P.rowq + h);  // filled right after the push
+                if (v == 0) *error = 1;
+                b = v - 1;
+                __threadfence();
+            }
+        }
+    }
+    return __shfl_sync(0xffffffffu, b, 0);
+}
+
 template <typename T>
 __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared& sh, int lane) {
     volatile int* error = &sh.error;
@@ -506,28 +539,20 @@ __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared&
             }
             if (__shfl_sync(0xffffffffu, *reinterpret_cast<volatile int*>(&sh.total_segs), 0) == sigma) own_done = true;
         }
-        // ---- duty 2: a completed batch row from the global queue
-        int b = -1;  // -1: queue empty; -2: lost the claim to another warp, look again
-        if (lane == 0) {
-            const int h = ld_volatile(P.qhead);
-            if (h < ld_volatile(P.qtail)) {
-                b = -2;
-                if (atomicCAS(P.qhead, h, h + 1) == h) {
-                    int v = 0;
-                    for (int it = 0; it < kWaitLimit && v == 0; ++it) v = ld_volatile(P.rowq + h);  // filled right after the push
-                    if (v == 0) *error = 1;
-                    b = v - 1;
-                    __threadfence();
-                }
-            }
+        // ---- duty 2: a completed batch row from the global queue.  Once the producer has issued
+        // everything, publishing must not be held up any more: the consumer warps, idle by then,
+        // take the remaining rows.
+        if (own_done) {
+            if (lane == 0) *reinterpret_cast<volatile int*>(&sh.published) = 1;
+            return;
         }
-        b = __shfl_sync(0xffffffffu, b, 0);
+        const bool tail = __shfl_sync(0xffffffffu, *reinterpret_cast<volatile int*>(&sh.total_segs), 0) >= 0;
+        const int b = tail ? -1 : pipe_pop_row(P, error, lane);
         if (b >= 0) {
             pipe_row_job<T>(P, sh, b, lane);
             idle = 0;
             continue;
         }
-        if (own_done && b == -1) return;  // nothing left of our own and nothing queued
         ++idle;
     }
     *error = 1;
@@ -535,7 +560,7 @@ __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared&
 
 // ---- the kernel -------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(kPipeThreads, 2) pipe_sweep_kernel(const __grid_constant__ KParams P) {
+__global__ void __launch_bounds__(kPipeThreads, SPECKV_PIPE_CTAS) pipe_sweep_kernel(const __grid_constant__ KParams P) {
     extern __shared__ __align__(128) unsigned char pipe_smem[];
     PipeShared& sh = *reinterpret_cast<PipeShared*>(pipe_smem);
     unsigned char* ring = pipe_smem + (sizeof(PipeShared) + 127) / 128 * 128;
@@ -546,6 +571,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) pipe_sweep_kernel(const __gri
         for (int s = 0; s < kSegSlots; ++s) { mbar_init(&sh.seg_bar[s], kPipeWarps); mbar_init(&sh.slot_free[s], 1); }
         sh.error = 0;
         sh.total_segs = -1;
+        sh.published = 0;
         sh.prefix[0] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -617,7 +643,7 @@ __global__ void __launch_bounds__(kPipeThreads, 2) pipe_sweep_kernel(const __gri
             return;
         }
         const StageDesc d = sh.desc[s];
-        if (d.flags & ST_END) return;
+        if (d.flags & ST_END) break;
         const uint4* stage = reinterpret_cast<const uint4*>(ring + static_cast<size_t>(s) * kStageBytes);
         if (d.flags & ST_FIRST) {
             const SegInfo& si = sh.seg[d.seg % kSegSlots];
@@ -644,6 +670,25 @@ __global__ void __launch_bounds__(kPipeThreads, 2) pipe_sweep_kernel(const __gri
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sh.empty[s]);
+    }
+    // The stream is used up: this warp now runs row epilogues from the global queue until its
+    // CTA has published all its segments and the queue is empty.  A row is queued by the warp that
+    // publishes its last segment, so the consumer warps of that CTA are still here to take it.
+    // (Two warps per CTA are plenty for the few rows left at that point, and keep the queue's
+    // counters from being polled by thousands of warps.)
+    if (warp >= 2) return;
+    for (int idle = 0; idle < kWaitLimit; ++idle) {
+        if (__shfl_sync(0xffffffffu, *error, 0)) return;
+        int published = 0;
+        if (lane == 0) {
+            published = *reinterpret_cast<volatile int*>(&sh.published);
+            __threadfence();  // the flag is read before the queue: whatever was queued before it was set is seen
+        }
+        published = __shfl_sync(0xffffffffu, published, 0);
+        const int b = pipe_pop_row(P, error, lane);
+        if (b >= 0) { pipe_row_job<T>(P, sh, b, lane); idle = 0; }
+        else if (b == -1 && published) return;
+        else __nanosleep(b == -2 ? 50 : 200);
     }
 }
 
