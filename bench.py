@@ -3,8 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload b256]
 
-A step = one pass of the whole hot path (draft signals, controller, verification: memset +
-sweep kernel + resample kernel) over one synthetic batch whose logits are resident in HBM.
+A step = one pass of the whole hot path (draft signals, controller, verification: a memset of the
+tickets, the sweep kernel and the resample kernel) over one synthetic batch whose logits are
+resident in HBM.
 Prints ONE JSON line: verified speculation rows/s (whole job), the roofline of the dominant
 kernel against the measured HBM peak, the end-to-end figure with host buffers, and the CPU
 oracle timed on the host cores as a reported baseline.  With --impl reference the oracle
@@ -53,9 +54,9 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def ncu_traffic_bytes(workload: str):
-    """DRAM bytes per sweep launch from the committed ncu summary, if there is one."""
-    p = os.path.join(ROOT, "profiles", f"sweep_kernel_{workload}.txt")
+def ncu_traffic_bytes(kernel: str, workload: str):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, if there is one."""
+    p = os.path.join(ROOT, "profiles", f"{kernel}_{workload}.txt")
     try:
         with open(p) as f:
             for line in f:
@@ -128,7 +129,17 @@ def run_reference(args, w):
     if rank != 0:
         return
     cores = host_cores()
-    rows = min(w.B, max(cores, 16))
+    # rows per step: sized from a short calibration so that warm-up + timed steps take about two minutes at most
+    cal_rows = min(w.B, max(cores, 16))
+    wc = synth.scaled(w, B=cal_rows)
+    sc = synth.make_step(wc, 0, "cpu")
+    mc = synth.make_mlp(wc, "cpu")
+    t0 = time.perf_counter()
+    oracle.step(oracle_batch(sc, n_threads=cores), sc["comp"].numpy(),
+                oracle.Mlp(*(mc[k].numpy() for k in ("W1", "b1", "W2", "b2"))))
+    rate = cal_rows / max(time.perf_counter() - t0, 1e-6)
+    budget_s = 120.0
+    rows = int(max(8, min(w.B, rate * budget_s / max(1, args.steps + args.warmup))))
     ws = synth.scaled(w, B=rows)
     s = synth.make_step(ws, 0, "cpu")
     mw = synth.make_mlp(ws, "cpu")
@@ -256,8 +267,9 @@ def main():
     bytes_avg = sum(bytes_step[i % n_batches] for i in range(n_prof)) / n_prof
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_avg / (sweep_avg * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "sweep_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(w.name),
+    kernel = "pipe_sweep_kernel" if w.dtype == "fp32" else "sweep_kernel"  # the library picks by logit type
+    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,
                 "algorithmic_bytes_per_launch": bytes_avg, "kernel_ms": sweep_avg,
                 "kernel_ms_min": min(sweep_ms), "resample_kernel_ms": sum(resample_ms) / n_prof,
                 "timed_over": f"{n_prof} steps after the timed region, CUDA events recorded inside the library call",
@@ -313,16 +325,20 @@ def main():
         import oracle
         from parity import oracle_batch
         cores = host_cores()
-        rows = list(range(min(w.B, 4 * max(cores, 8))))
-        ob = oracle_batch(steps_in[0], rows=rows, n_threads=cores)
+        # bounded sample: whole batches of the resident steps, repeated until about 12 s of CPU work
+        # are done (rows per batch capped so that one call stays near a second)
+        rows = list(range(min(w.B, 256)))
+        obs = [oracle_batch(s_, rows=rows, n_threads=cores) for s_ in steps_in]
         mw = synth.make_mlp(wr, "cpu")
         om = oracle.Mlp(*(mw[k2].numpy() for k2 in ("W1", "b1", "W2", "b2")))
-        comp = steps_in[0]["comp"].cpu().numpy()[rows]
-        t0 = time.perf_counter()
-        oracle.step(ob, comp, om)
+        comps = [s_["comp"].cpu().numpy()[rows] for s_ in steps_in]
+        calls, t0 = 0, time.perf_counter()
+        while calls < 3 or (time.perf_counter() - t0 < 12.0 and calls < 200):
+            oracle.step(obs[calls % n_batches], comps[calls % n_batches], om)
+            calls += 1
         dt = time.perf_counter() - t0
-        cpu_baseline = {"value": len(rows) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-                        "sample": f"first {len(rows)} rows of step 0 of workload {w.name}, one call, {dt:.2f} s"}
+        cpu_baseline = {"value": calls * len(rows) / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"{calls} calls of {len(rows)} rows (steps 0/1 of workload {w.name} in turn), {dt:.1f} s"}
 
     if rank == 0:
         gam = steps_in[0]["gamma"]

@@ -514,9 +514,14 @@ __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared&
             const int ready = __shfl_sync(0xffffffffu, mbar_test(&sh.seg_bar[slot], (sigma / kSegSlots) & 1) ? 1 : 0, 0);
             if (ready) {
                 const SegInfo si = sh.seg[slot];
-                float4 acc = sh.part[slot][lane & (kPipeWarps - 1)];
+                // lanes beyond the consumer warps start from an empty partial of the segment's kind
+                float4 acc = (si.path == PATH_TARGET) ? make_float4(-3.0e38f, 0.f, 0.f, 0.f)
+                           : (si.path == PATH_DRAFT) ? make_float4(kFloor, 0.f, 0.f, 0.f)
+                                                     : make_float4(kFloor, __int_as_float(0x7fffffff), 0.f, 0.f);
+                if (lane < kPipeWarps) acc = sh.part[slot][lane];
+                static_assert(kPipeWarps <= 16, "the merge tree below spans 16 lanes");
 #pragma unroll
-                for (int o = kPipeWarps / 2; o > 0; o >>= 1) {
+                for (int o = 8; o > 0; o >>= 1) {
                     const float4 other = shfl_xor4(acc, o);
                     acc = (si.path == PATH_DRAFT) ? merge_draft(acc, other, si.scale)
                         : (si.path == PATH_TARGET) ? merge_target(acc, other) : merge_argmax(acc, other);

@@ -119,6 +119,35 @@ def test_b256_full_batch_sampled_rows():
     assert set(np.unique(out["gamma_next"].cpu().numpy())) <= {2, 4, 6, 8}
 
 
+def test_b512_mixed_full_batch_sampled_rows():
+    # fp32 logits at full size: the bulk-copy ring sweep in the configuration the benchmark can time
+    w = synth.WORKLOADS["b512_mixed"]
+    attrs = synth.row_attrs(w)
+    greedy = np.nonzero(attrs.temperature.numpy() == 0)[0]
+    hot = np.nonzero(attrs.onehot.numpy())[0]
+    rows = np.unique(np.concatenate([[0, 1, 255, 256, 510, 511], greedy[:2], hot[:2]]))
+    s, out, ref = _run_both(w, rows=rows, attrs=attrs)
+    compare_step(out, ref, rows=rows)
+    n = out["n_accepted"].cpu().numpy(); g = s["gamma"].cpu().numpy()
+    assert np.all((n >= 0) & (n <= g)) and np.all(out["row_status"].cpu().numpy() == 0)
+    H = out["H"].cpu().numpy(); C = out["C"].cpu().numpy()
+    assert np.all(H >= 0) and np.all(H <= math.log(w.V) + 1e-4) and np.all(C <= 1.0 + 1e-6)
+    ot = out["out_tokens"].cpu().numpy()
+    assert np.all(ot[np.arange(w.B), n] >= 0) and np.all(ot[np.arange(w.B), n] < w.V)
+
+
+def test_batches_beyond_the_ring_sweep_table_take_the_other_kernel():
+    # more rows than the staged sweep's per-row tables hold: same results from the register-staged kernel
+    w = synth.Workload("t", B=1100, gamma_max=2, V=512, dtype="fp32", gamma_mode="ragged", temperature=0.9,
+                       sigma_d=synth.SIGMA_LEVELS, seed=12)
+    rows = np.array([0, 1, 511, 1023, 1024, 1099])
+    s, out, ref = _run_both(w, rows=rows)
+    compare_step(out, ref, rows=rows)
+    w2 = synth.scaled(w, B=1024)   # the largest batch the ring sweep takes
+    s, out, ref = _run_both(w2, rows=rows[:4])
+    compare_step(out, ref, rows=rows[:4])
+
+
 # ---- separate entry points ----
 def test_signals_verify_and_controller_entry_points_agree_with_step():
     w = synth.Workload("t", B=12, gamma_max=5, V=9000, dtype="bf16", gamma_mode="ragged", temperature=0.7,
