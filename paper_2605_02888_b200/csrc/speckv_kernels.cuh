@@ -1143,8 +1143,10 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     asm volatile("griddepcontrol.wait;" ::: "memory");
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
-    const int b = blockIdx.x / P.R;
-    const int share = blockIdx.x - b * P.R;
+    // (last batch row first: the sweep touched those rows most recently, part of them is still in L2)
+    const int bq = blockIdx.x / P.R;
+    const int share = blockIdx.x - bq * P.R;
+    const int b = P.B - 1 - bq;
     const RowInfo ri = P.info[b];
     if (ri.mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
 
