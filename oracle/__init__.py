@@ -155,9 +155,16 @@ class Mlp:
         W2 = np.ascontiguousarray(self.W2, np.float32)
         b2 = np.ascontiguousarray(self.b2, np.float32)
         m = _Mlp()
-        m.n_hidden, m.n_in = W1.shape
-        m.n_out = W2.shape[0]
-        assert W2.shape[1] == m.n_hidden and b1.shape == (m.n_hidden,) and b2.shape == (m.n_out,)
+        if self.feature_layout == 2:
+            # the paper's f(x, gamma): one output, evaluated per candidate; W1 [0, n_in] => linear
+            m.n_hidden, m.n_in = W1.shape
+            m.n_out = len(self.gamma_choices)
+            assert W2.shape == (1, m.n_hidden if m.n_hidden else m.n_in) and b2.shape == (1,)
+            assert b1.shape == (m.n_hidden,) and m.n_out <= 8
+        else:
+            m.n_hidden, m.n_in = W1.shape
+            m.n_out = W2.shape[0]
+            assert W2.shape[1] == m.n_hidden and b1.shape == (m.n_hidden,) and b2.shape == (m.n_out,)
         assert len(self.gamma_choices) >= m.n_out
         m.W1, m.b1, m.W2, m.b2 = W1.ctypes.data, b1.ctypes.data, W2.ctypes.data, b2.ctypes.data
         for j in range(m.n_out):
@@ -167,7 +174,11 @@ class Mlp:
 
     @property
     def n_comp(self) -> int:
-        return self.W1.shape[1] - (3 if self.feature_layout == 0 else 4)
+        return self.W1.shape[1] - (3, 4, 5)[self.feature_layout]
+
+    @property
+    def n_out(self) -> int:
+        return len(self.gamma_choices) if self.feature_layout == 2 else self.W2.shape[0]
 
 
 def signals(bt: Batch):

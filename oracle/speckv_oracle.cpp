@@ -223,9 +223,62 @@ void signals_row(const oracle_batch* bt, int32_t b, double* H, double* C, double
     }
 }
 
+/* compression entries per row: what is left of n_in after the signals (and the gamma input) */
+inline int32_t n_comp_of(const oracle_mlp* mlp) {
+    return mlp->n_in - (mlp->feature_layout == 0 ? 3 : mlp->feature_layout == 1 ? 4 : 5);
+}
+
+/* ---- controller in the paper's own form (Sec. 4.3): one predictor f(x, gamma) -> a_hat with
+ * x = [Hbar, cbar, Hmax, cmin, comp...] and the candidate gamma as the last input, evaluated once
+ * per candidate; E = a_hat * gamma + 1 (Eq. 1); gamma* = argmax.  n_hidden = 0 is the linear
+ * (Ridge) predictor: a_hat = W2 . [x, gamma] + b2. ---- */
+void select_gamma_row_paper_form(const double* feat4, const float* comp, const oracle_mlp* mlp, double* scores,
+                                 int32_t* gamma_next, int32_t* near) {
+    const int32_t n_in = mlp->n_in;
+    std::vector<double> x(n_in, 0.0);
+    for (int32_t k = 0; k < 4; ++k) x[k] = feat4[k];
+    for (int32_t k = 4; k < n_in - 1; ++k) x[k] = comp ? static_cast<double>(comp[k - 4]) : 0.0;
+    int32_t best = 0;
+    double best_e = 0.0, second_e = -std::numeric_limits<double>::infinity();
+    for (int32_t j = 0; j < mlp->n_out; ++j) {
+        x[n_in - 1] = static_cast<double>(mlp->gamma_choices[j]);
+        double a_hat = static_cast<double>(mlp->b2[0]);
+        if (mlp->n_hidden == 0) {
+            for (int32_t f = 0; f < n_in; ++f) a_hat += static_cast<double>(mlp->W2[f]) * x[f];
+        } else {
+            for (int32_t k = 0; k < mlp->n_hidden; ++k) {
+                double a = static_cast<double>(mlp->b1[k]);
+                for (int32_t f = 0; f < n_in; ++f)
+                    a += static_cast<double>(mlp->W1[static_cast<int64_t>(k) * n_in + f]) * x[f];
+                if (a > 0.0) a_hat += static_cast<double>(mlp->W2[k]) * a;
+            }
+        }
+        const double e = (mlp->score_transform == 0) ? a_hat * mlp->gamma_choices[j] + 1.0 : a_hat;
+        if (scores) scores[j] = e;
+        if (j == 0) {
+            best_e = e;
+        } else if (e > best_e) {
+            second_e = best_e;
+            best_e = e;
+            best = j;
+        } else if (e > second_e) {
+            second_e = e;
+        }
+    }
+    if (gamma_next) *gamma_next = mlp->gamma_choices[best];
+    if (near) {
+        bool tie = (mlp->n_out > 1) && (best_e - second_e) < 1e-5 * std::max(std::fabs(best_e), 1e-30);
+        if (tie) *near |= ORACLE_NEAR_GAMMA;
+    }
+}
+
 /* ---- controller, one row (paper Sec. 4.3, Eq. 1) ---- */
 void select_gamma_row(const double* feat4, const float* comp, const oracle_mlp* mlp, double* scores,
                       int32_t* gamma_next, int32_t* near) {
+    if (mlp->feature_layout == 2) {
+        select_gamma_row_paper_form(feat4, comp, mlp, scores, gamma_next, near);
+        return;
+    }
     std::vector<double> x(mlp->n_in, 0.0);
     if (mlp->feature_layout == 0) {
         /* mean entropy, mean confidence, min confidence, two compression flags */
@@ -411,10 +464,10 @@ int oracle_signals(const oracle_batch* bt, double* H, double* C, double* feat, i
 
 int oracle_select_gamma(int32_t B, const double* feat, const float* comp, const oracle_mlp* mlp,
                         double* scores, int32_t* gamma_next, int32_t* near) {
-    if (B < 0 || !mlp || !feat || mlp->n_out < 1 || mlp->n_out > 8 || mlp->n_hidden < 1 ||
-        mlp->n_in < 4)
-        return 1;
-    const int32_t n_comp = mlp->n_in - (mlp->feature_layout == 0 ? 3 : 4);
+    if (B < 0 || !mlp || !feat || mlp->n_out < 1 || mlp->n_out > 8 || mlp->n_in < 4) return 1;
+    if (mlp->n_hidden < (mlp->feature_layout == 2 ? 0 : 1)) return 1;
+    if (mlp->feature_layout == 2 && mlp->n_in < 5) return 1;
+    const int32_t n_comp = n_comp_of(mlp);
     for (int32_t b = 0; b < B; ++b)
         select_gamma_row(feat + static_cast<int64_t>(b) * 4,
                          comp ? comp + static_cast<int64_t>(b) * n_comp : nullptr, mlp,
@@ -439,7 +492,7 @@ int oracle_step(const oracle_batch* bt, const float* comp, const oracle_mlp* mlp
     if (!batch_ok(bt, true) || !mlp || !feat || !n_accepted || !out_tokens || !row_status) return 1;
     std::fill(row_status, row_status + bt->B, 0);
     if (near) std::fill(near, near + bt->B, 0);
-    const int32_t n_comp = mlp->n_in - (mlp->feature_layout == 0 ? 3 : 4);
+    const int32_t n_comp = n_comp_of(mlp);
     for_rows(bt->B, bt->n_threads, [&](int32_t b) {
         signals_row(bt, b, H, C, feat, row_status);
         verify_row(bt, b, n_accepted, out_tokens, row_status, near);

@@ -66,7 +66,10 @@ typedef struct {
     const float* W2;               /* [n_out, n_hidden]                                   */
     const float* b2;               /* [n_out]                                             */
     int32_t gamma_choices[8];      /* first n_out entries used                            */
-    int32_t feature_layout;        /* 0: [Hbar,cbar,cmin,flag0,flag1]; 1: [Hbar,cbar,Hmax,cmin,comp] */
+    int32_t feature_layout;        /* 0: [Hbar,cbar,cmin,flag0,flag1]; 1: [Hbar,cbar,Hmax,cmin,comp];
+                                      2: the paper's f(x, gamma): [Hbar,cbar,Hmax,cmin,comp..,gamma_j], one
+                                         output (W2 [1,n_hidden], b2 [1]) evaluated for each of the n_out
+                                         candidates; n_hidden = 0: linear predictor, W2 [1,n_in]        */
     int32_t score_transform;       /* 0: E_j = o_j*gamma_j + 1 (Eq. 1); 1: E_j = o_j      */
 } oracle_mlp;
 

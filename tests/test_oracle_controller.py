@@ -93,3 +93,47 @@ def test_random_network_matches_numpy_matmul(layout, n_comp):
     E = o * np.array([2, 4, 6, 8]) + 1
     np.testing.assert_allclose(r["scores"], E, rtol=1e-12)
     np.testing.assert_array_equal(r["gamma_next"], np.array([2, 4, 6, 8])[E.argmax(1)])
+
+
+# ---- the paper's own predictor form (Sec. 4.3): f(x, gamma) -> a_hat, evaluated per candidate ----
+def test_paper_form_linear_predictor_closed_form():
+    # a_hat(gamma) = 0.5 - 0.06 gamma  =>  E(gamma) = gamma (0.5 - 0.06 gamma) + 1, maximal near 0.5 / 0.12 = 4.17
+    feat = np.array([[1.0, 0.5, 2.0, 0.25]])
+    comp = np.array([[1.0]], np.float32)
+    W2 = np.array([[0.1, 0.2, 0.0, 0.4, -0.1, -0.06]], np.float32)       # [Hbar, cbar, Hmax, cmin, comp, gamma]
+    m = oracle.Mlp(np.zeros((0, 6), np.float32), np.zeros(0, np.float32), W2, np.array([0.3], np.float32),
+                   feature_layout=2)
+    out = oracle.select_gamma(feat, comp, m)
+    want = [g * (0.5 - 0.06 * g) + 1.0 for g in (2, 4, 6, 8)]
+    np.testing.assert_allclose(out["scores"][0], want, rtol=1e-6)
+    assert out["gamma_next"][0] == 4
+    raw = oracle.select_gamma(feat, comp, oracle.Mlp(m.W1, m.b1, m.W2, m.b2, feature_layout=2, score_transform=1))
+    # (weights are float32: the cancellation at gamma = 8 leaves an absolute 1e-8, not a relative 1e-6)
+    np.testing.assert_allclose(raw["scores"][0], [0.5 - 0.06 * g for g in (2, 4, 6, 8)], rtol=1e-6, atol=1e-7)
+
+
+def test_paper_form_hidden_units_by_hand():
+    # h1 = relu(Hbar + gamma - 5), h2 = relu(7 - gamma); a_hat = 0.1 h1 + 0.05 h2; Hbar = 1
+    feat = np.array([[1.0, 0.0, 0.0, 0.0]])
+    W1 = np.array([[1, 0, 0, 0, 0, 1], [0, 0, 0, 0, 0, -1]], np.float32)
+    b1 = np.array([-5, 7], np.float32)
+    W2 = np.array([[0.1, 0.05]], np.float32)
+    m = oracle.Mlp(W1, b1, W2, np.array([0.0], np.float32), feature_layout=2)
+    out = oracle.select_gamma(feat, np.zeros((1, 1), np.float32), m)
+    a_hat = np.array([0.25, 0.15, 0.25, 0.4])
+    np.testing.assert_allclose(out["scores"][0], a_hat * np.array([2, 4, 6, 8]) + 1.0, rtol=1e-6)
+    assert out["gamma_next"][0] == 8
+
+
+def test_paper_form_without_gamma_dependence_picks_an_end_of_the_range():
+    rng = np.random.default_rng(3)
+    feat = np.abs(rng.normal(size=(50, 4)))
+    comp = rng.integers(0, 3, (50, 1)).astype(np.float32)
+    W1 = rng.normal(0, 0.3, (16, 6)).astype(np.float32)
+    W1[:, 5] = 0                                                          # the prediction ignores gamma
+    m = oracle.Mlp(W1, rng.normal(0, 0.3, 16).astype(np.float32), rng.normal(0, 0.3, (1, 16)).astype(np.float32),
+                   np.array([0.01], np.float32), feature_layout=2)
+    out = oracle.select_gamma(feat, comp, m)
+    a_hat = (out["scores"][:, 0] - 1.0) / 2.0
+    assert np.all(out["gamma_next"][a_hat > 1e-6] == 8) and np.all(out["gamma_next"][a_hat < -1e-6] == 2)
+    np.testing.assert_allclose(out["scores"], a_hat[:, None] * np.array([2, 4, 6, 8]) + 1.0, rtol=1e-9, atol=1e-12)
