@@ -96,6 +96,11 @@ typedef struct {
     int32_t gamma_choices[8];      /* candidate gammas, first n_out used ({2,4,6,8})      */
     int32_t feature_layout;        /* 0: x = [Hbar, cbar, cmin, comp0, comp1]             */
                                    /* 1: x = [Hbar, cbar, Hmax, cmin, comp0] (Sec. 4.3)   */
+                                   /* 2: the predictor exactly as Sec. 4.3 writes it,      */
+                                   /*    a_hat = f([Hbar, cbar, Hmax, cmin, comp.., gamma_j]): one */
+                                   /*    output (W2 [1,n_hidden], b2 [1]) evaluated for each of the */
+                                   /*    n_out candidate gammas; n_hidden = 0 makes it the linear  */
+                                   /*    (Ridge) predictor with W2 [1,n_in], W1 and b1 unused      */
     int32_t score_transform;       /* 0: E_j = o_j * gamma_j + 1 (Eq. 1); 1: E_j = o_j    */
 } speckv_mlp;
 
@@ -111,7 +116,7 @@ speckv_status speckv_signals(const speckv_batch* batch, float* H, float* C, floa
                              void* cuda_stream);
 
 /* Controller (paper Sec. 4.3, Eq. 1).  feat: [B,4] as written by speckv_signals;
- * comp: [B, n_in-3] (layout 0) or [B, n_in-4] (layout 1) fp32, NULL => zeros;
+ * comp: [B, n_in-3] (layout 0), [B, n_in-4] (layout 1) or [B, n_in-5] (layout 2) fp32, NULL => zeros;
  * scores: [B, n_out] fp32 (may be NULL); gamma_next: [B] int32.  Ties go to the
  * lowest candidate index.                                                                 */
 speckv_status speckv_select_gamma(int32_t B, const float* feat, const float* comp,

@@ -176,17 +176,22 @@ class Mlp:
 
     @property
     def n_out(self):
-        return self.W2.shape[0]
+        # layout 2 (the paper's f(x, gamma)): one head, one score per candidate gamma
+        return len(self.gamma_choices) if self.feature_layout == 2 else self.W2.shape[0]
 
     @property
     def n_comp(self):
-        return self.n_in - (3 if self.feature_layout == 0 else 4)
+        return self.n_in - (3, 4, 5)[self.feature_layout]
 
     def _c(self) -> _CMlp:
         m = _CMlp()
         m.n_hidden, m.n_in = self.W1.shape
-        m.n_out = self.W2.shape[0]
-        if self.W2.shape[1] != m.n_hidden or tuple(self.b1.shape) != (m.n_hidden,) or tuple(self.b2.shape) != (m.n_out,):
+        m.n_out = self.n_out
+        if self.feature_layout == 2:
+            if tuple(self.W2.shape) != (1, m.n_hidden if m.n_hidden else m.n_in) or tuple(self.b2.shape) != (1,) \
+                    or tuple(self.b1.shape) != (m.n_hidden,):
+                raise ValueError("inconsistent controller shapes for the paper-form predictor")
+        elif self.W2.shape[1] != m.n_hidden or tuple(self.b1.shape) != (m.n_hidden,) or tuple(self.b2.shape) != (m.n_out,):
             raise ValueError("inconsistent controller shapes")
         if len(self.gamma_choices) < m.n_out or m.n_out > 8:
             raise ValueError("need one gamma choice per output (at most 8)")

@@ -88,12 +88,14 @@ speckv_status check_batch(const speckv_batch* bt, bool need_target) {
 }
 
 speckv_status check_mlp(const speckv_mlp* m) {
-    if (!m || !m->W1 || !m->b1 || !m->W2 || !m->b2) return SPECKV_ERR_INVALID_ARG;
-    if (m->n_hidden < 1 || m->n_out < 1 || m->n_in < 1) return SPECKV_ERR_INVALID_ARG;
+    if (!m || !m->W2 || !m->b2) return SPECKV_ERR_INVALID_ARG;
+    if (m->feature_layout < 0 || m->feature_layout > 2) return SPECKV_ERR_INVALID_ARG;
+    const int min_hidden = m->feature_layout == 2 ? 0 : 1;  // the paper-form predictor may be linear
+    if (m->n_hidden < min_hidden || m->n_out < 1 || m->n_in < 1) return SPECKV_ERR_INVALID_ARG;
+    if (m->n_hidden > 0 && (!m->W1 || !m->b1)) return SPECKV_ERR_INVALID_ARG;
     if (m->n_hidden > SPECKV_MAX_HIDDEN || m->n_out > 8 || m->n_in > 8) return SPECKV_ERR_UNSUPPORTED;
-    if (m->feature_layout != 0 && m->feature_layout != 1) return SPECKV_ERR_INVALID_ARG;
     if (m->score_transform != 0 && m->score_transform != 1) return SPECKV_ERR_INVALID_ARG;
-    if (m->n_in < (m->feature_layout == 0 ? 3 : 4)) return SPECKV_ERR_INVALID_ARG;
+    if (m->n_in < (m->feature_layout == 0 ? 3 : m->feature_layout == 1 ? 4 : 5)) return SPECKV_ERR_INVALID_ARG;
     return SPECKV_OK;
 }
 
@@ -104,7 +106,7 @@ bool rows_aligned(const void* base, int64_t sb, int64_t sp, int es) {
 void fill_mlp(KParams& P, const speckv_mlp* m, const float* comp) {
     P.n_in = m->n_in; P.n_hidden = m->n_hidden; P.n_out = m->n_out;
     P.layout = m->feature_layout; P.transform = m->score_transform;
-    P.n_comp = m->n_in - (m->feature_layout == 0 ? 3 : 4);
+    P.n_comp = m->n_in - (m->feature_layout == 0 ? 3 : m->feature_layout == 1 ? 4 : 5);
     P.W1 = m->W1; P.b1 = m->b1; P.W2 = m->W2; P.b2 = m->b2; P.comp = comp;
     for (int j = 0; j < 8; ++j) P.gch[j] = m->gamma_choices[j];
 }

@@ -653,10 +653,18 @@ __device__ __forceinline__ CtlRegs ctl_load(const KParams& P, int b, int lane) {
     const bool hid = lane < P.n_hidden;
 #pragma unroll
     for (int f = 0; f < 8; ++f) c.w1[f] = (hid && f < P.n_in) ? __ldg(P.W1 + lane * P.n_in + f) : 0.f;
+    if (P.layout == 2) {
+        // the paper's f(x, gamma): one output head; without hidden units W2 weighs the inputs directly
 #pragma unroll
-    for (int j = 0; j < 8; ++j) c.w2[j] = (hid && j < P.n_out) ? __ldg(P.W2 + j * P.n_hidden + lane) : 0.f;
+        for (int j = 1; j < 8; ++j) c.w2[j] = 0.f;
+        c.w2[0] = (P.n_hidden > 0 ? hid : lane < P.n_in) ? __ldg(P.W2 + lane) : 0.f;
+        c.b2k = lane == 0 ? __ldg(P.b2) : 0.f;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) c.w2[j] = (hid && j < P.n_out) ? __ldg(P.W2 + j * P.n_hidden + lane) : 0.f;
+        c.b2k = lane < P.n_out ? __ldg(P.b2 + lane) : 0.f;
+    }
     c.b1 = hid ? __ldg(P.b1 + lane) : 0.f;
-    c.b2k = lane < P.n_out ? __ldg(P.b2 + lane) : 0.f;
     c.compk = (P.comp && lane < P.n_comp) ? __ldg(P.comp + static_cast<long long>(b) * P.n_comp + lane) : 0.f;
     return c;
 }
@@ -664,6 +672,45 @@ __device__ __forceinline__ CtlRegs ctl_load(const KParams& P, int b, int lane) {
 __device__ __forceinline__ void ctl_eval(const KParams& P, const CtlRegs& c, const float (&f4)[4],
                                          float* scores_row, int* gamma_next) {
     const int lane = threadIdx.x & 31;
+    if (P.layout == 2) {
+        // Sec. 4.3 as printed: a_hat = f([Hbar, cbar, Hmax, cmin, comp.., gamma_j]) for every candidate
+        float x[8];
+        x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[2]; x[3] = f4[3];
+#pragma unroll
+        for (int k = 4; k < 8; ++k) {
+            const float cv = __shfl_sync(0xffffffffu, c.compk, k - 4);
+            x[k] = (k < P.n_in - 1) ? cv : 0.f;
+        }
+        float base = c.b1, wg = 0.f, xl = 0.f;  // hidden pre-activation without gamma; gamma's weight; x[lane]
+#pragma unroll
+        for (int f = 0; f < 8; ++f) {
+            if (f < P.n_in - 1) base = fmaf(c.w1[f], x[f], base);
+            if (f == P.n_in - 1) wg = c.w1[f];
+            if (f == lane) xl = x[f];
+        }
+        const float b2 = __shfl_sync(0xffffffffu, c.b2k, 0);
+        float best = 0.f;
+        int best_j = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < P.n_out) {  // uniform across the warp
+                const float g = static_cast<float>(P.gch[j]);
+                float term;
+                if (P.n_hidden > 0) {
+                    const float h = fmaf(wg, g, base);
+                    term = (lane < P.n_hidden && h > 0.f) ? c.w2[0] * h : 0.f;
+                } else {
+                    term = lane < P.n_in - 1 ? c.w2[0] * xl : (lane == P.n_in - 1 ? c.w2[0] * g : 0.f);
+                }
+                const float a_hat = warp_sumf(term) + b2;
+                const float e = (P.transform == 0) ? fmaf(a_hat, g, 1.f) : a_hat;
+                if (scores_row && lane == 0) scores_row[j] = e;
+                if (j == 0 || e > best) { best = e; best_j = j; }
+            }
+        }
+        if (gamma_next && lane == 0) *gamma_next = P.gch[best_j];
+        return;
+    }
     float x[8];
     const int first_comp = (P.layout == 0) ? 3 : 4;
     if (P.layout == 0) { x[0] = f4[0]; x[1] = f4[1]; x[2] = f4[3]; x[3] = 0.f; }

@@ -192,6 +192,35 @@ def test_paper_form_controller_layout():
         assert not (bad & ((ref["near"] & oracle.NEAR_GAMMA) == 0)).any()
 
 
+def test_paper_form_predictor_per_candidate_gamma():
+    # Sec. 4.3 as printed: one predictor f(x, gamma) -> a_hat, evaluated for every candidate gamma
+    rng = np.random.default_rng(1)
+    feat = torch.tensor(np.abs(rng.normal(size=(200, 4))), dtype=torch.float32, device=DEV)
+    comp = torch.tensor(rng.integers(0, 3, (200, 1)), dtype=torch.float32, device=DEV)
+    t = lambda a: torch.tensor(a, dtype=torch.float32, device=DEV)
+    mlp16 = dict(W1=t(rng.normal(0, 0.3, (16, 6))), b1=t(rng.normal(0, 0.3, 16)), W2=t(rng.normal(0, 0.3, (1, 16))),
+                 b2=t(rng.normal(0, 0.1, 1)))
+    ridge = dict(W1=torch.zeros(0, 6, device=DEV), b1=torch.zeros(0, device=DEV), W2=t(rng.normal(0, 0.2, (1, 6))),
+                 b2=t([0.4]))
+    for w in (mlp16, ridge):
+        for kw in (dict(feature_layout=2), dict(feature_layout=2, score_transform=1)):
+            gm, om = mlp_pair(w, **kw)
+            out = speckv.speckv_select_gamma(feat, comp, gm)
+            ref = oracle.select_gamma(feat.cpu().numpy().astype(np.float64), comp.cpu().numpy(), om)
+            assert out["scores"].shape == (200, 4)
+            close(out["scores"].cpu().numpy(), ref["scores"], "scores", atol=2e-7)
+            bad = out["gamma_next"].cpu().numpy() != ref["gamma_next"]
+            assert not (bad & ((ref["near"] & oracle.NEAR_GAMMA) == 0)).any()
+    # and inside the fused step
+    wl = synth.Workload("t", B=10, gamma_max=4, V=3000, dtype="fp32", gamma_mode="ragged", sigma_d=(0.5,), seed=2)
+    s = synth.make_step(wl, 0, DEV)
+    gm, om = mlp_pair(mlp16, feature_layout=2)
+    comp1 = s["comp"][:, :1].contiguous()
+    out = speckv.speckv_step(gpu_batch(s), comp1, gm)
+    ref = oracle.step(oracle_batch(s), comp1.cpu().numpy(), om)
+    compare_step(out, ref)
+
+
 # ---- edge cases ----
 def _small(dtype="fp32", B=6, G=3, V=600, seed=0):
     w = synth.Workload("e", B=B, gamma_max=G, V=V, dtype=dtype, gamma_mode="fixed", gamma_fixed=G,
