@@ -23,15 +23,6 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kVec = 8;                 // elements per lane per step
 constexpr int kChunk = 32 * kVec;       // one warp step = one inverse-CDF chunk (256 elements)
 constexpr int kMaxSplit = 32;
-#ifndef SPECKV_WARP_RANGES
-#define SPECKV_WARP_RANGES 0  // 1: each warp streams its own contiguous range; 0: the CTA's threads interleave
-#endif
-#ifndef SPECKV_PACKED
-#define SPECKV_PACKED 1       // 1: f32x2 packed arithmetic in the sweep; 0: scalar fp32
-#endif
-#ifndef SPECKV_SYNC_WARM
-#define SPECKV_SYNC_WARM 1    // 1: CTA barrier before reading the other warps' warm-start maxima; 0: read what is there
-#endif
 #ifndef SPECKV_U
 #define SPECKV_U 4            // 16-byte loads in flight per thread (bf16); fp32 uses half as many vector steps
 #endif
@@ -339,23 +330,6 @@ struct DraftState {
             return;
         }
         raw_floor(raw);
-#if !SPECKV_PACKED
-        {
-            float xs[kVec];
-            unpack<T>(raw, xs);
-            float z0, z1, z2, z3, s0, s1, s2, s3;
-            unpack2(za, z0, z1); unpack2(zb, z2, z3); unpack2(sa, s0, s1); unpack2(sb, s2, s3);
-#pragma unroll
-            for (int j = 0; j < kVec; j += 4) {
-                float d0 = xs[j] - m, d1 = xs[j + 1] - m, d2 = xs[j + 2] - m, d3 = xs[j + 3] - m;
-                float e0 = ex2f(d0 * scale), e1 = ex2f(d1 * scale), e2 = ex2f(d2 * scale), e3 = ex2f(d3 * scale);
-                z0 += e0; z1 += e1; z2 += e2; z3 += e3;
-                s0 = fmaf(e0, d0, s0); s1 = fmaf(e1, d1, s1); s2 = fmaf(e2, d2, s2); s3 = fmaf(e3, d3, s3);
-            }
-            za = pack2(z0, z1); zb = pack2(z2, z3); sa = pack2(s0, s1); sb = pack2(s2, s3);
-            return;
-        }
-#endif
         f2 x[4];
         unpack_pairs(raw, x);
         const f2 m2 = pack2(m, m), sc2 = pack2(scale, scale);
@@ -407,21 +381,6 @@ struct TargetState {
                 r = rn; m = vmax;
             }
         }
-#if !SPECKV_PACKED
-        {
-            float xs[kVec];
-            unpack<T>(raw, xs);
-            float z0, z1, z2, z3;
-            unpack2(za, z0, z1); unpack2(zb, z2, z3);
-#pragma unroll
-            for (int j = 0; j < kVec; j += 4) {
-                z0 += ex2f(fmaf(xs[j], scale, -r)); z1 += ex2f(fmaf(xs[j + 1], scale, -r));
-                z2 += ex2f(fmaf(xs[j + 2], scale, -r)); z3 += ex2f(fmaf(xs[j + 3], scale, -r));
-            }
-            za = pack2(z0, z1); zb = pack2(z2, z3);
-            return;
-        }
-#endif
         f2 x[4];
         unpack_pairs(raw, x);
         const f2 sc2 = pack2(scale, scale), nr2 = pack2(-r, -r);
@@ -572,15 +531,9 @@ __device__ __forceinline__ float4 sweep_warp(const T* __restrict__ row, int lo, 
         if (v >= kFloor && v < __int_as_float(0x7f800000)) m0 = fmaxf(m0, v);
     }
     m0 = warp_maxf(m0);
-    // share the warm start across the CTA's warps: publish ours, take what the others have
-    // published so far (slots start at the floor).  Nobody waits; a late warp only costs the
-    // readers a few more trips through the slow path.
+    // share the warm start across the CTA's warps (one barrier per CTA, before the streaming loop)
     if ((threadIdx.x & 31) == 0) sh_m0[threadIdx.x >> 5] = m0;
-#if SPECKV_SYNC_WARM
     __syncthreads();
-#else
-    __syncwarp();
-#endif
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) m0 = fmaxf(m0, sh_m0[w]);
 
@@ -949,22 +902,11 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
         // the CTA's slice of the row
         const int v0 = s * P.per_split;
         const int v1 = min(P.nvec, v0 + P.per_split);
-#if SPECKV_WARP_RANGES
-        // one contiguous range per warp (whole warp-steps)
-        constexpr int STEP = 32;
-        const int first = lane;
-        const int per_warp = (((v1 - v0) + kWarps - 1) / kWarps + 31) / 32 * 32;
-        const int wv0 = min(v1, v0 + warp * per_warp);
-        const int wv1 = min(v1, wv0 + per_warp);
-        const int lo = wv0 * kVec;
-        const int hi = min(P.V, wv1 * kVec);
-#else
         // the CTA's threads interleave over the slice: consecutive warps read consecutive 512 bytes
         constexpr int STEP = kThreads;
         const int first = threadIdx.x;
         const int lo = v0 * kVec;
         const int hi = min(P.V, v1 * kVec);
-#endif
         float4 part;
         int path;
         if (is_target) {
