@@ -67,6 +67,8 @@ def lib():
                                           C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_verify.restype = C.c_int
         L.oracle_verify.argtypes = [C.POINTER(_Batch), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_sample_draft.restype = C.c_int
+        L.oracle_sample_draft.argtypes = [C.POINTER(_Batch)] + [C.c_void_p] * 4
         L.oracle_step.restype = C.c_int
         L.oracle_step.argtypes = [C.POINTER(_Batch), C.c_void_p, C.POINTER(_Mlp)] + [C.c_void_p] * 9
         L.oracle_softmax_row.restype = C.c_int
@@ -214,6 +216,18 @@ def verify(bt: Batch):
     if rc:
         raise ValueError("oracle_verify: invalid arguments")
     return dict(n_accepted=n, out_tokens=out, row_status=st, near=near)
+
+
+def sample_draft(bt: Batch, uniforms: np.ndarray):
+    """tokens[b,i] ~ softmax(draft[b,i] / T_b) by inverse CDF at uniforms[b,i]; argmax for T_b = 0."""
+    c, keep = bt._c()
+    B, G = c.B, c.gamma_max
+    u = np.ascontiguousarray(uniforms, np.float32).reshape(B, G)
+    tok = np.zeros((B, G), np.int32); st = np.zeros(B, np.int32); near = np.zeros(B, np.int32)
+    rc = lib().oracle_sample_draft(C.byref(c), _ptr(u), _ptr(tok), _ptr(st), _ptr(near))
+    if rc:
+        raise ValueError("oracle_sample_draft: invalid arguments")
+    return dict(tokens=tok, row_status=st, near=near)
 
 
 def step(bt: Batch, comp: Optional[np.ndarray], mlp: Mlp):

@@ -486,6 +486,42 @@ int oracle_verify(const oracle_batch* bt, int32_t* n_accepted, int32_t* out_toke
     return 0;
 }
 
+/* Drafting (paper Sec. 3.1: the draft model proposes gamma tokens): position i of row b draws its
+ * token from q_i = softmax(d[b,i] / T_b) by the same inverse-CDF convention as the verification
+ * draws (vocabulary order, threshold u * sum); T_b = 0 takes the argmax (lowest index). */
+int oracle_sample_draft(const oracle_batch* bt, const float* uniforms, int32_t* tokens,
+                        int32_t* row_status, int32_t* near) {
+    if (!batch_ok(bt, false) || !tokens || !uniforms) return 1;
+    const int32_t G = bt->gamma_max, V = bt->V;
+    if (row_status) std::fill(row_status, row_status + bt->B, 0);
+    if (near) std::fill(near, near + bt->B, 0);
+    for_rows(bt->B, bt->n_threads, [&](int32_t b) {
+        int32_t* tb = tokens + static_cast<int64_t>(b) * G;
+        std::fill(tb, tb + G, -1);
+        const RowParams rp = row_params(bt, b);
+        int32_t status = rp.status;
+        std::vector<int32_t> tok(G, -1);
+        std::vector<double> q(V);
+        int32_t nearbits = 0;
+        for (int32_t i = 0; !status && i < rp.gamma; ++i) {
+            if (rp.T == 0.0) {
+                const RowRef r = draft_row(bt, b, i);
+                if (!softmax_row(r, V, 1.0, q.data())) { status |= ORACLE_ROW_NONFINITE; break; }
+                tok[i] = argmax_row(r, V);
+            } else {
+                if (!softmax_row(draft_row(bt, b, i), V, rp.T, q.data())) { status |= ORACLE_ROW_NONFINITE; break; }
+                int32_t nb = 0;
+                tok[i] = inverse_cdf(q.data(), V, static_cast<double>(uniforms[static_cast<int64_t>(b) * G + i]), &nb);
+                if (nb) nearbits |= ORACLE_NEAR_CDF;
+            }
+        }
+        if (!status) std::copy(tok.begin(), tok.end(), tb);
+        if (row_status) row_status[b] = status;
+        if (near) near[b] = nearbits;
+    });
+    return 0;
+}
+
 int oracle_step(const oracle_batch* bt, const float* comp, const oracle_mlp* mlp, double* H,
                 double* C, double* feat, double* scores, int32_t* gamma_next,
                 int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status, int32_t* near) {

@@ -86,6 +86,12 @@ int oracle_select_gamma(int32_t B, const double* feat, const float* comp, const 
 int oracle_verify(const oracle_batch* bt, int32_t* n_accepted, int32_t* out_tokens,
                   int32_t* row_status, int32_t* near);
 
+/* Drafting: tokens[b,i] ~ softmax(draft[b,i] / T_b) for i < gamma_b by inverse CDF at
+ * uniforms[b,i] (vocabulary order); argmax for T_b = 0; -1 at i >= gamma_b and in flagged rows.
+ * uniforms: [B, gamma_max] floats.  tokens: [B, gamma_max].  near: [B] or NULL.             */
+int oracle_sample_draft(const oracle_batch* bt, const float* uniforms, int32_t* tokens,
+                        int32_t* row_status, int32_t* near);
+
 /* Whole step = signals -> controller -> verification on one batch. */
 int oracle_step(const oracle_batch* bt, const float* comp, const oracle_mlp* mlp, double* H,
                 double* C, double* feat, double* scores, int32_t* gamma_next,
