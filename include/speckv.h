@@ -130,6 +130,17 @@ speckv_status speckv_verify(const speckv_batch* batch, int32_t* n_accepted, int3
                             int32_t* row_status, void* workspace, size_t workspace_bytes,
                             void* cuda_stream);
 
+/* Drafting (paper Sec. 3.1: the draft model proposes gamma tokens): tokens[b,i] for i < gamma_b is
+ * drawn from softmax(draft_logits[b,i] / T_b) by inverse CDF in vocabulary order at
+ * uniforms[b,i] (the convention of the verification draws); T_b = 0 takes the argmax (lowest
+ * index).  tokens: [B, gamma_max] int32, -1 at i >= gamma_b and in flagged rows; uniforms:
+ * [B, gamma_max] fp32 in [0,1); row_status may be NULL.  Reads only the draft logits, gamma and
+ * temperature.  Needs its own scratch size (one resample slot per drafted position).          */
+speckv_status speckv_sample_workspace_size(const speckv_batch* batch, size_t* bytes);
+speckv_status speckv_sample_draft(const speckv_batch* batch, const float* uniforms, int32_t* tokens,
+                                  int32_t* row_status, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream);
+
 /* One fused step: signals, controller and verification from a single pass over the logits
  * (plus a second look at the stop position's two rows for the residual / bonus draw).
  * gamma_next[b] is the controller's choice for the NEXT step of row b; this step verifies

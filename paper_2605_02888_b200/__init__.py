@@ -1,9 +1,9 @@
 """SpecKV speculation-step hot path for B200 (sm_100a): draft signals, gamma controller and
 draft verification from one pass over vocabulary-sized logits, behind a C ABI (libspeckv)."""
-from .binding import (Batch, Mlp, StepOutputs, SpeckvError, load_library, speckv_select_gamma,
+from .binding import (Batch, Mlp, StepOutputs, SpeckvError, load_library, speckv_sample_draft, speckv_select_gamma,
                       speckv_signals, speckv_signals_static, speckv_step, speckv_verify, status_string, version,
                       workspace_size)
 
-__all__ = ["Batch", "Mlp", "StepOutputs", "SpeckvError", "load_library", "speckv_select_gamma",
+__all__ = ["Batch", "Mlp", "StepOutputs", "SpeckvError", "load_library", "speckv_sample_draft", "speckv_select_gamma",
            "speckv_signals", "speckv_signals_static", "speckv_step", "speckv_verify", "status_string", "version",
            "workspace_size"]

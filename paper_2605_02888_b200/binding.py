@@ -22,6 +22,7 @@ ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE, ROW_TI
 
 STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_signals_static", "speckv_select_gamma", "speckv_verify",
+           "speckv_sample_workspace_size", "speckv_sample_draft",
            "speckv_step", "speckv_step_profiled", "speckv_status_string", "speckv_version")
 
 
@@ -71,6 +72,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_signals.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, vp, sz, vp]
     L.speckv_signals_static.restype = C.c_int
     L.speckv_signals_static.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, vp]
+    L.speckv_sample_workspace_size.restype = C.c_int
+    L.speckv_sample_workspace_size.argtypes = [C.POINTER(_CBatch), C.POINTER(sz)]
+    L.speckv_sample_draft.restype = C.c_int
+    L.speckv_sample_draft.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, sz, vp]
     L.speckv_select_gamma.restype = C.c_int
     L.speckv_select_gamma.argtypes = [C.c_int32, vp, vp, C.POINTER(_CMlp), vp, vp, vp]
     L.speckv_verify.restype = C.c_int
@@ -286,6 +291,35 @@ def speckv_signals_static(batch: Batch, H: torch.Tensor, Cc: torch.Tensor, feat:
     if rc != OK:
         raise SpeckvError(rc, "speckv_signals_static")
     return dict(H=H, C=Cc, feat=feat, row_status=row_status)
+
+
+def speckv_sample_draft(batch: Batch, uniforms: torch.Tensor, tokens: Optional[torch.Tensor] = None,
+                        row_status: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """Draft tokens (paper Sec. 3.1): tokens[b,i] ~ softmax(draft_logits[b,i] / T_b) by inverse CDF at
+    uniforms[b,i] (argmax for T_b = 0); -1 beyond gamma_b.  uniforms: [B, gamma_max] fp32."""
+    L = load_library()
+    c = batch._c()
+    B, G, V = batch.shape()
+    dev = batch.draft_logits.device
+    if tuple(uniforms.shape) != (B, G):
+        raise ValueError(f"uniforms must have shape {(B, G)}")
+    if tokens is None:
+        tokens = torch.empty(B, G, dtype=torch.int32, device=dev)
+    if row_status is None:
+        row_status = torch.empty(B, dtype=torch.int32, device=dev)
+    if workspace is None:
+        n = C.c_size_t(0)
+        rc = L.speckv_sample_workspace_size(C.byref(c), C.byref(n))
+        if rc != OK:
+            raise SpeckvError(rc, "speckv_sample_workspace_size")
+        workspace = torch.empty(int(n.value), dtype=torch.uint8, device=dev)
+    with torch.cuda.device(dev):
+        rc = L.speckv_sample_draft(C.byref(c), _dev_ptr(uniforms, torch.float32, "uniforms"),
+                                   _dev_ptr(tokens, torch.int32, "tokens"), _dev_ptr(row_status, torch.int32, "row_status"),
+                                   _ptr(workspace), workspace.numel(), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_sample_draft")
+    return dict(tokens=tokens, row_status=row_status)
 
 
 def speckv_select_gamma(feat: torch.Tensor, comp: Optional[torch.Tensor], mlp: Mlp,

@@ -248,6 +248,79 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 
+// Draft-side sampling: its own workspace plan (one resample slot per drafted position).
+struct SamplePlan {
+    int nchunk, R, chunks_per_cta;
+    size_t off_tick, off_info, off_part, off_csum, total;
+};
+SamplePlan make_sample_plan(const speckv_batch* bt) {
+    SamplePlan p;
+    const size_t B = static_cast<size_t>(bt->B), G = static_cast<size_t>(bt->gamma_max);
+    p.nchunk = (bt->V + kChunk - 1) / kChunk;
+    p.R = (p.nchunk + 63) / 64;
+    if (p.R > 32) p.R = 32;
+    if (p.R < 1) p.R = 1;
+    p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
+    size_t off = 0;
+    p.off_tick = off; off = align_up(off + (B + B * G) * sizeof(int));  // sweep tickets, resample tickets
+    p.off_info = off; off = align_up(off + B * G * sizeof(RowInfo));
+    p.off_part = off; off = align_up(off + B * G * kMaxSplit * sizeof(float4));
+    p.off_csum = off; off = align_up(off + B * G * p.nchunk * sizeof(float));
+    p.total = off < kAlign ? kAlign : off;
+    return p;
+}
+
+speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t* tokens, int32_t* row_status,
+                         void* ws, size_t ws_bytes, void* stream) {
+    speckv_status st = check_batch(bt, false);
+    if (st != SPECKV_OK) return st;
+    if (bt->B == 0) return SPECKV_OK;
+    if (!uniforms || !tokens) return SPECKV_ERR_INVALID_ARG;
+    if (static_cast<long long>(bt->B) * bt->gamma_max > (1 << 24)) return SPECKV_ERR_UNSUPPORTED;
+    const SamplePlan pl = make_sample_plan(bt);
+    if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SPECKV_ERR_INVALID_ARG;
+    if (ws_bytes < pl.total) return SPECKV_ERR_WORKSPACE;
+
+    KParams P{};
+    P.B = bt->B; P.G = bt->gamma_max; P.V = bt->V;
+    P.J = bt->gamma_max;
+    P.nsplit = choose_nsplit(P.B, P.J, P.V, bt->dtype);
+    P.nvec = (bt->V + kVec - 1) / kVec;
+    P.per_split = (P.nvec + P.nsplit - 1) / P.nsplit;
+    P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
+    P.mode = MODE_SAMPLE; P.sample = 1;
+    // the drafted positions are swept and drawn from as if they were target rows
+    P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
+    P.t = bt->draft_logits; P.tsb = bt->draft_stride_b; P.tsp = bt->draft_stride_pos;
+    P.gamma = bt->gamma; P.temp = bt->temperature; P.temp_scalar = bt->temperature_scalar;
+    P.u = uniforms;
+    P.out_tok = tokens; P.status = row_status;
+    char* w = static_cast<char*>(ws);
+    P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
+    P.tick2 = P.tick1 + P.B;
+    P.info = reinterpret_cast<RowInfo*>(w + pl.off_info);
+    P.part = reinterpret_cast<float4*>(w + pl.off_part);
+    P.csum = reinterpret_cast<float*>(w + pl.off_csum);
+    if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const size_t n_tick = static_cast<size_t>(P.B) * (1 + static_cast<size_t>(P.G));
+    if (cudaMemsetAsync(P.tick1, 0, n_tick * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+    const int es = esize(bt->dtype);
+    const bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
+    const unsigned grid1 = static_cast<unsigned>(P.B) * P.J * P.nsplit;
+    const unsigned grid2 = static_cast<unsigned>(P.B) * P.G * P.R;
+    constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
+    if (bt->dtype == SPECKV_BF16) {
+        if (aligned) { sweep_kernel<__nv_bfloat16, true, Ub><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<__nv_bfloat16, true><<<grid2, kThreads, 0, cs>>>(P); }
+        else { sweep_kernel<__nv_bfloat16, false, Ub><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<__nv_bfloat16, false><<<grid2, kThreads, 0, cs>>>(P); }
+    } else {
+        if (aligned) { sweep_kernel<float, true, Uf><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<float, true><<<grid2, kThreads, 0, cs>>>(P); }
+        else { sweep_kernel<float, false, Uf><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<float, false><<<grid2, kThreads, 0, cs>>>(P); }
+    }
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
 // Scratch for speckv_signals_static: lives in the library image, one copy per device that loads it.
 static __device__ __align__(256) unsigned char g_static_scratch[SPECKV_STATIC_SCRATCH_BYTES];
 
@@ -298,6 +371,21 @@ speckv_status speckv_signals_static(const speckv_batch* batch, float* H, float* 
     // run() clears the ticket counters on the caller's stream; nothing else needs a known start
     return run(batch, MODE_SIGNALS, nullptr, nullptr, H, C, feat, nullptr, nullptr, nullptr, nullptr,
                row_status, scratch, SPECKV_STATIC_SCRATCH_BYTES, cuda_stream);
+}
+
+speckv_status speckv_sample_workspace_size(const speckv_batch* batch, size_t* bytes) {
+    if (!bytes) return SPECKV_ERR_INVALID_ARG;
+    if (!batch || batch->B < 0 || batch->gamma_max < 1 || batch->V < 1) return SPECKV_ERR_INVALID_ARG;
+    if (batch->gamma_max > SPECKV_MAX_GAMMA || batch->V > (1 << 30) || batch->B > (1 << 24))
+        return SPECKV_ERR_UNSUPPORTED;
+    *bytes = make_sample_plan(batch).total;
+    return SPECKV_OK;
+}
+
+speckv_status speckv_sample_draft(const speckv_batch* batch, const float* uniforms, int32_t* tokens,
+                                  int32_t* row_status, void* workspace, size_t workspace_bytes,
+                                  void* cuda_stream) {
+    return run_sample(batch, uniforms, tokens, row_status, workspace, workspace_bytes, cuda_stream);
 }
 
 speckv_status speckv_select_gamma(int32_t B, const float* feat, const float* comp,

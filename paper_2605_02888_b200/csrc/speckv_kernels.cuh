@@ -34,7 +34,7 @@ constexpr uint32_t kFloorBf16x2 = 0xF180F180u;     // -2^100 as two bf16
 constexpr double kLn2 = 0.6931471805599453094;
 constexpr double kLog2e = 1.4426950408889634074;
 
-enum : int { MODE_SIGNALS = 1, MODE_VERIFY = 2, MODE_MLP = 4 };
+enum : int { MODE_SIGNALS = 1, MODE_VERIFY = 2, MODE_MLP = 4, MODE_SAMPLE = 8 };
 enum : int { PATH_DRAFT = 0, PATH_TARGET = 1, PATH_ARGMAX = 2 };
 enum : int { RS_NONE = 0, RS_RESIDUAL = 1, RS_BONUS = 2 };
 
@@ -49,6 +49,7 @@ struct RowInfo {  // written by the sweep kernel's row epilogue, read by the res
 
 struct KParams {
     int B, G, V, J, nsplit, nvec, per_split, nchunk, R, chunks_per_cta, mode, bits;
+    int sample;  // 1: draft-side sampling (every drafted position draws a token from its own row)
     int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
     const void* t; long long tsb, tsp;
@@ -865,6 +866,49 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     if (P.status && lane == 0) P.status[b] = status;
 }
 
+// Epilogue of the draft-side sampling sweep (one warp per batch row): lane i merges the partials
+// of drafted position i into the row's log2-normaliser (or its argmax for a greedy row) and leaves
+// one RowInfo per position for the resample kernel, which then draws from softmax(d_i / T).
+__device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pt, int nt) {
+    const int lane = threadIdx.x & 31;
+    const int G = P.G;
+    int status = 0;
+    if (gam < 1 || gam > G) status |= 1;
+    if (!(Tf >= 0.f) || Tf == __int_as_float(0x7f800000)) status |= 8;
+    const bool greedy = (Tf == 0.f);
+    const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
+    const bool on = !status && lane < gam;
+    double lse2 = 0.0;
+    int amax = -1;
+    bool nonfinite = false;
+    if (on) {
+        float4 at = ldcg4(pt);
+        for (int k = 1; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
+        if (greedy) {
+            amax = __float_as_int(at.y);
+            if (at.z != 0.f || amax == 0x7fffffff || !(at.x > kFloor)) nonfinite = true;
+        } else {
+            if (!(at.y > 0.f) || !(at.y < 3e38f)) nonfinite = true;
+            else lse2 = static_cast<double>(at.x) + log2_split(static_cast<double>(at.y));
+        }
+    }
+    if (__any_sync(0xffffffffu, nonfinite)) status |= 4;
+    if (lane < G) {
+        const long long r = static_cast<long long>(b) * G + lane;
+        const bool ok = (status == 0 && lane < gam);
+        RowInfo ri;
+        ri.mode = (ok && !greedy) ? RS_BONUS : RS_NONE;
+        ri.n = lane;
+        ri.u2 = (ok && !greedy) ? __ldg(P.u + r) : 0.f;
+        ri.scale = scale;
+        ri.lse2_p = lse2;
+        ri.lse2_q = 0.0;
+        P.info[r] = ri;
+        P.out_tok[r] = (ok && greedy) ? amax : -1;
+    }
+    if (P.status && lane == 0) P.status[b] = status;
+}
+
 // ----------------------------------------------------------------------------------------
 // Sweep kernel
 // ----------------------------------------------------------------------------------------
@@ -894,9 +938,11 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
 
     // logit row handled by this CTA: with verification, j <= G are target positions and the
     // rest draft positions; signals alone sweep draft positions only
-    const bool is_target = verify && j <= P.G;
+    // (draft-side sampling sweeps the drafted positions with the target statistics: only the
+    // normaliser, or the argmax, of each row is needed; P.t then points at the draft logits)
+    const bool is_target = P.sample || (verify && j <= P.G);
     const int pos = is_target ? j : (verify ? j - (P.G + 1) : j);
-    const bool active = row_ok && (is_target ? pos <= gam : pos < gam);
+    const bool active = row_ok && ((is_target && !P.sample) ? pos <= gam : pos < gam);
 
     if (active) {
         // the CTA's slice of the row
@@ -952,6 +998,10 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
     if (!__shfl_sync(0xffffffffu, last_row, 0)) return;
     __threadfence();
     const long long row0 = static_cast<long long>(b) * P.J;
+    if (P.sample) {
+        sample_epilogue(P, b, gam, Tf, P.part + (row0 + lane) * P.nsplit, P.nsplit);
+        return;
+    }
     row_epilogue<T>(P, b, gam, Tf, P.part + (row0 + (verify ? P.G + 1 + lane : lane)) * P.nsplit, P.nsplit,
                     P.part + (row0 + lane) * P.nsplit, P.nsplit);
 }
@@ -1133,17 +1183,21 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
     // (last batch row first: the sweep touched those rows most recently, part of them is still in L2)
+    // (draft-side sampling: one draw per drafted position; r counts positions, b = r / gamma_max)
+    const int n_draws = P.sample ? P.B * P.G : P.B;
     const int bq = blockIdx.x / P.R;
     const int share = blockIdx.x - bq * P.R;
-    const int b = P.B - 1 - bq;
-    const RowInfo ri = P.info[b];
+    const int r = n_draws - 1 - bq;
+    const int b = P.sample ? r / P.G : r;
+    const RowInfo ri = P.info[r];
     if (ri.mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
+    const long long out_at = P.sample ? static_cast<long long>(r) : static_cast<long long>(b) * (P.G + 1) + ri.n;
 
     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
                     static_cast<long long>(ri.n) * P.tsp;
     const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb +
                     static_cast<long long>(ri.n) * P.dsp;
-    float* csum = P.csum + static_cast<long long>(b) * P.nchunk;
+    float* csum = P.csum + static_cast<long long>(r) * P.nchunk;
     RsConst c = rs_const(ri, ri.mode);
 
     const int c0 = share * P.chunks_per_cta;
@@ -1153,7 +1207,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
-        int old = atomicAdd(P.tick2 + b, 1);
+        int old = atomicAdd(P.tick2 + r, 1);
         sh_flag = (old == P.R - 1);
     }
     __syncthreads();
@@ -1173,7 +1227,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     if (sh_empty) {
         // numerically empty residual (p == q at the stop position): draw from p instead
         if (c.mode != RS_RESIDUAL) {  // p itself has no mass: cannot happen for a finite row
-            if (threadIdx.x == 0) P.out_tok[static_cast<long long>(b) * (P.G + 1) + ri.n] = 0;
+            if (threadIdx.x == 0) P.out_tok[out_at] = 0;
             return;
         }
         c.mode = RS_BONUS;
@@ -1244,7 +1298,7 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
     }
     if (lane == 0) {
         int tok = (found != 0x7fffffff) ? found : lastw;
-        P.out_tok[static_cast<long long>(b) * (P.G + 1) + ri.n] = tok;
+        P.out_tok[out_at] = tok;
     }
 }
 

@@ -221,6 +221,43 @@ def test_paper_form_predictor_per_candidate_gamma():
     compare_step(out, ref)
 
 
+# ---- draft-side sampling ----
+@pytest.mark.parametrize("dtype,V", [("bf16", 128256), ("fp32", 4099), ("bf16", 33)])
+def test_sample_draft_against_oracle(dtype, V):
+    w = synth.Workload("t", B=20, gamma_max=5, V=V, dtype=dtype, gamma_mode="ragged", temperature_mode="mixed",
+                       sigma_d=(0.5,), seed=31)
+    s = synth.make_step(w, 0, DEV)
+    u = torch.rand(w.B, w.gamma_max, device=DEV)
+    u[0, 0] = 0.0
+    out = speckv.speckv_sample_draft(gpu_batch(s), u)
+    ref = oracle.sample_draft(oracle_batch(s), u.cpu().numpy())
+    tok = out["tokens"].cpu().numpy()
+    np.testing.assert_array_equal(out["row_status"].cpu().numpy(), ref["row_status"])
+    bad = (tok != ref["tokens"]).any(1)
+    assert not (bad & ((ref["near"] & oracle.NEAR_CDF) == 0)).any()
+    g = s["gamma"].cpu().numpy()
+    cols = np.arange(w.gamma_max)[None, :]
+    assert np.all(tok[cols >= g[:, None]] == -1) and np.all(tok[cols < g[:, None]] >= 0)
+    assert (s["temperature"] == 0).any() and (s["temperature"] > 0).any()
+
+
+def test_sample_draft_distribution_and_flags():
+    rng = np.random.default_rng(8)
+    V, N, T = 8, 200_000, 0.9
+    row = torch.tensor(rng.normal(0, 1.4, (1, V)), dtype=torch.float32, device=DEV)
+    u = torch.rand(N, 1, device=DEV)
+    out = speckv.speckv_sample_draft(speckv.Batch(draft_logits=row[None].expand(N, 1, V), temperature_scalar=T), u)
+    q = torch.softmax(row[0].double() / float(np.float32(T)), -1).cpu().numpy()
+    cnt = np.bincount(out["tokens"].cpu().numpy()[:, 0], minlength=V)
+    assert scipy.stats.chisquare(cnt, q * N).pvalue > 1e-4
+    d = torch.zeros(3, 2, 64, device=DEV)
+    d[1, 1, 7] = float("nan")
+    gam = torch.tensor([2, 2, 0], dtype=torch.int32, device=DEV)
+    out = speckv.speckv_sample_draft(speckv.Batch(draft_logits=d, gamma=gam), torch.rand(3, 2, device=DEV))
+    assert out["row_status"].tolist() == [0, 4, 1]
+    assert out["tokens"][1:].flatten().tolist() == [-1] * 4 and (out["tokens"][0] >= 0).all()
+
+
 # ---- edge cases ----
 def _small(dtype="fp32", B=6, G=3, V=600, seed=0):
     w = synth.Workload("e", B=B, gamma_max=G, V=V, dtype=dtype, gamma_mode="fixed", gamma_fixed=G,
