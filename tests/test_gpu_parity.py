@@ -354,8 +354,32 @@ def test_gamma_max_16_and_strided_views():
     compare_step(out3, ref)
 
 
-def test_results_are_deterministic():
-    w = synth.scaled(synth.WORKLOADS["b256"], B=16)
+def test_ring_sweep_with_padded_rows_and_ragged_ends_fp32():
+    # fp32 logits in a wider buffer: rows 16-byte aligned but not adjacent, V not a multiple of a block
+    w = synth.Workload("e", B=5, gamma_max=6, V=5004, dtype="fp32", gamma_mode="ragged", temperature_mode="mixed",
+                       sigma_d=(0.4,), seed=14)
+    s = synth.make_step(w, 0, DEV)
+    gm, om = mlp_pair(synth.make_mlp(w, DEV))
+    ref = oracle.step(oracle_batch(s), s["comp"].cpu().numpy(), om)
+    out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
+    compare_step(out, ref)
+    pt = torch.full((w.B, w.gamma_max + 2, 5120), 3.0, device=DEV)
+    pd = torch.full((w.B, w.gamma_max + 1, 5120), 3.0, device=DEV)
+    pt[:, 1:w.gamma_max + 2, :w.V] = s["target"]; pd[:, :w.gamma_max, :w.V] = s["draft"]
+    s2 = dict(s); s2["target"] = pt[:, 1:w.gamma_max + 2, :w.V]; s2["draft"] = pd[:, :w.gamma_max, :w.V]
+    out2 = speckv.speckv_step(gpu_batch(s2), s["comp"], gm)
+    for k in out:
+        assert torch.equal(out[k], out2[k]), k
+    # an element offset of one breaks the 16-byte alignment: the register-staged kernel's element-wise path
+    flat = torch.zeros(s["target"].numel() + 1, device=DEV)
+    flat[1:] = s["target"].flatten()
+    s3 = dict(s); s3["target"] = flat[1:].view_as(s["target"])
+    compare_step(speckv.speckv_step(gpu_batch(s3), s["comp"], gm), ref)
+
+
+@pytest.mark.parametrize("name", ["b256", "b512_mixed"])
+def test_results_are_deterministic(name):
+    w = synth.scaled(synth.WORKLOADS[name], B=16)
     s = synth.make_step(w, 0, DEV)
     gm, _ = mlp_pair(synth.make_mlp(w, DEV))
     a = {k: v.clone() for k, v in speckv.speckv_step(gpu_batch(s), s["comp"], gm).items()}
