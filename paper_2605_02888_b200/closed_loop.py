@@ -24,25 +24,32 @@ from . import binding as speckv
 from . import synth
 
 
-def run(w: synth.Workload, steps: int, device, policy: str = "controller", gamma_fixed: int = 4) -> Dict:
-    """Run `steps` speculation steps of workload `w`; returns tokens/step statistics and the gamma
-    histogram of the last step.  policy: "controller" (gamma_next feeds the next step) or "fixed"."""
+def run(w: synth.Workload, steps: int, device, policy: str = "controller", gamma_fixed: int = 4,
+        mlp: "speckv.Mlp" = None, first_step: int = 0) -> Dict:
+    """Run `steps` speculation steps of workload `w` (stream steps first_step, first_step+1, ...);
+    returns tokens/step statistics and the gamma histogram of the last step.  policy: "controller"
+    (gamma_next feeds the next step) or "fixed".  mlp: the controller to use (default: the
+    workload's own random draw, primary 5 -> 16 -> 4 form)."""
     if policy not in ("controller", "fixed"):
         raise ValueError("policy must be 'controller' or 'fixed'")
     attrs = synth.row_attrs(w)
-    mw = synth.make_mlp(w, device)
-    mlp = speckv.Mlp(mw["W1"], mw["b1"], mw["W2"], mw["b2"])
+    if mlp is None:
+        mw = synth.make_mlp(w, device)
+        mlp = speckv.Mlp(mw["W1"], mw["b1"], mw["W2"], mw["b2"])
+    # the paper-form predictor takes one compression scalar (0 / 1 / 2), the primary form two flags
+    comp_scalar = (attrs.comp[:, 0] + 2 * attrs.comp[:, 1]).reshape(-1, 1).contiguous().to(device)
     gamma = torch.full((w.B,), min(gamma_fixed, w.gamma_max), dtype=torch.int32, device=device)
     emitted = torch.zeros(w.B, dtype=torch.int64, device=device)
     drafted = torch.zeros(w.B, dtype=torch.int64, device=device)
     out = None
-    for step in range(steps):
+    for step in range(first_step, first_step + steps):
         s = synth.make_step(w, step, device, attrs=attrs, gamma=gamma)
+        comp = s["comp"] if mlp.feature_layout == 0 else comp_scalar
         bt = speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],
                           gamma=s["gamma"], temperature=s["temperature"], uniforms=s["uniforms"])
         if out is None:
             out = speckv.StepOutputs.allocate(bt, mlp.n_out)
-        res = speckv.speckv_step(bt, s["comp"], mlp, out=out)
+        res = speckv.speckv_step(bt, comp, mlp, out=out)
         if int(res["row_status"].abs().sum()) != 0:
             raise RuntimeError("a row was flagged during the closed-loop run")
         emitted += res["n_accepted"].to(torch.int64) + 1
