@@ -26,7 +26,7 @@ struct Plan {
     int nchunk;      // 256-element chunks per logit row
     int R;           // resample CTAs per batch row
     int chunks_per_cta;
-    size_t off_tick, off_info, off_part, off_csum, total;
+    size_t off_tick, off_info, off_part, off_csum, off_tokl, total;
 };
 
 inline int esize(speckv_dtype dt) { return dt == SPECKV_BF16 ? 2 : 4; }
@@ -60,10 +60,11 @@ Plan make_plan(const speckv_batch* bt) {
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
     size_t off = 0;
-    p.off_tick = off; off = align_up(off + (3 * B + 4) * sizeof(int));  // tickets, counters, row queue
+    p.off_tick = off; off = align_up(off + (4 * B + 4) * sizeof(int));  // tickets, counters, row queue, row flags
     p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
     p.off_part = off; off = align_up(off + B * p.J_full * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
+    p.off_tokl = off; off = align_up(off + B * static_cast<size_t>(bt->gamma_max) * sizeof(float2));
     p.total = off < kAlign ? kAlign : off;
     return p;
 }
@@ -139,25 +140,35 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
     return cudaGetLastError();
 }
 
+// 1: after the register-staged sweep the fresh tokens are drawn by extra CTAs of the same launch;
+// 0: always by a second kernel (measurement builds)
+#ifndef SPECKV_MERGED
+#define SPECKV_MERGED 1
+#endif
+
 template <typename T, bool ALIGNED>
-cudaError_t launch_all(const KParams& P, cudaStream_t st, const Events& ev, bool staged) {
+cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged) {
     constexpr int U = sizeof(T) == 2 ? SPECKV_U : (SPECKV_U + 1) / 2;
-    const long long grid = static_cast<long long>(P.B) * P.J * P.nsplit;
+    const bool verify = (P.mode & MODE_VERIFY) != 0;
+    const bool ring = ALIGNED && staged;
+    const long long n_draw = static_cast<long long>(P.B) * P.R;
+    const bool merged = SPECKV_MERGED && verify && !ring && P.rdone && P.n_sweep + n_draw <= 0x7fffffffLL;
     if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
     cudaError_t e;
-    if (ALIGNED && staged) {
+    if (ring) {
         e = launch_pipe<T>(P, st);
     } else {
+        const long long grid = P.n_sweep + (merged ? n_draw : 0);
         sweep_kernel<T, ALIGNED, U><<<static_cast<unsigned>(grid), kThreads, 0, st>>>(P);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return e;
     if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
-    if (P.mode & MODE_VERIFY) {
+    if (verify && !merged) {
         // programmatic dependent launch: the kernel's CTAs are scheduled while the sweep drains and
         // wait inside the kernel for the sweep's results
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R));
+        cfg.gridDim = dim3(static_cast<unsigned>(n_draw));
         cfg.blockDim = dim3(kThreads);
         cfg.dynamicSmemBytes = 0;
         cfg.stream = st;
@@ -218,9 +229,10 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     P.csum = reinterpret_cast<float*>(w + pl.off_csum);
 
     if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+    P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(P.tick1, 0, (3 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
+    if (cudaMemsetAsync(P.tick1, 0, (4 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
 
     const int es = esize(bt->dtype);
@@ -238,6 +250,12 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
 #endif
     const bool staged = (SPECKV_STAGED == 2 || (SPECKV_STAGED == 1 && bt->dtype == SPECKV_F32)) && aligned &&
                         row_bytes % 16 == 0 && P.B <= kPipeMaxB;
+    // completion flags per batch row and the logits at the draft tokens: only the register-staged sweep
+    // overlaps the resample work with its own tail; after the ring sweep the resample kernel starts when
+    // everything is done and a flag would only cost it a round trip
+    P.rdone = (verify && !staged) ? P.rowq + P.B : nullptr;
+    P.tokl = (verify && !staged) ? reinterpret_cast<float2*>(static_cast<char*>(ws) + pl.off_tokl) : nullptr;
+    P.rs_reverse = staged ? 1 : 0;  // the ring sweep ends all at once: no drain for the resample kernel to fill
     P.Lg = static_cast<int>(row_bytes / 16);
     P.Lp = (P.Lg + kStageGran - 1) / kStageGran * kStageGran;
     cudaError_t e;
@@ -288,7 +306,7 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     P.nvec = (bt->V + kVec - 1) / kVec;
     P.per_split = (P.nvec + P.nsplit - 1) / P.nsplit;
     P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
-    P.mode = MODE_SAMPLE; P.sample = 1;
+    P.mode = MODE_SAMPLE; P.sample = 1; P.rs_reverse = 1;
     // the drafted positions are swept and drawn from as if they were target rows
     P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
     P.t = bt->draft_logits; P.tsb = bt->draft_stride_b; P.tsp = bt->draft_stride_pos;
@@ -302,6 +320,7 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     P.part = reinterpret_cast<float4*>(w + pl.off_part);
     P.csum = reinterpret_cast<float*>(w + pl.off_csum);
     if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+    P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const size_t n_tick = static_cast<size_t>(P.B) * (1 + static_cast<size_t>(P.G));

@@ -47,9 +47,13 @@ struct RowInfo {  // written by the sweep kernel's row epilogue, read by the res
     double lse2_q;  // same for the draft row (residual only)
 };
 
+static_assert(sizeof(RowInfo) == 32, "the resample kernel reads a RowInfo as two 16-byte words");
+
 struct KParams {
     int B, G, V, J, nsplit, nvec, per_split, nchunk, R, chunks_per_cta, mode, bits;
+    int n_sweep;  // sweep kernel: CTAs that sweep; the rest of the grid (if any) does the resample work
     int sample;  // 1: draft-side sampling (every drafted position draws a token from its own row)
+    int rs_reverse;  // resample kernel: 1 = last batch row first (after a sweep it cannot overlap: those rows are the freshest in L2)
     int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
     const void* t; long long tsb, tsp;
@@ -64,6 +68,8 @@ struct KParams {
     // workspace
     int *tick1, *tick2;
     int *qcount, *qhead, *qtail, *rowq;  // staged sweep: next quantum to hand out; queue of completed batch rows
+    float2* tokl;  // [B, G] (draft logit, target logit) at the draft token, left by the register-staged sweep; may be NULL
+    int* rdone;  // verification: rdone[b] = 1 once batch row b's epilogue has written everything the resample kernel reads
     RowInfo* info;
     float4* part;
     float* csum;
@@ -702,11 +708,34 @@ __device__ __forceinline__ double log2_split(double z) {
     return static_cast<double>(k) + static_cast<double>(log2f(static_cast<float>(m)));
 }
 
+// End of a row epilogue (whole warp): everything the warp wrote for batch row b becomes visible
+// before the row's completion flag does.  The resample kernel polls the flag instead of waiting for
+// the whole sweep grid, so it can work on finished rows while the sweep's last CTAs drain.
+__device__ __forceinline__ void row_done_signal(const KParams& P, int b) {
+    if (!P.rdone) return;
+    __threadfence();
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(P.rdone + b), "r"(1) : "memory");
+}
+
+// Bounded wait for a row's completion flag (one thread polls).  False when the bound ran out.
+__device__ __forceinline__ bool row_done_wait(const int* flag) {
+    for (int it = 0; it < (1 << 20); ++it) {
+        int v;
+        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v) return true;
+        __nanosleep(it < 64 ? 100 : 1000);
+    }
+    return false;
+}
+
 // Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
 // merges the nd partials at pd (draft position i) and the nt partials at pt (target position i).
 // gam and Tf are the row's gamma and temperature as the sweep read them.  Everything the row
 // needs from memory that does not depend on other loads is requested first, so the epilogue
-// costs two memory round trips (the second for the logits at the draft tokens).
+// costs one memory round trip (two when the sweep did not leave the logits at the draft tokens).
+// Order: what the resample kernel needs (acceptance, stop position, normalisers), the row's
+// completion flag, then the signals and the controller.
 template <typename T>
 __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd, int nd,
                                           const float4* pt, int nt) {
@@ -736,15 +765,18 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     const int x = tok_on ? __ldg(P.tok + static_cast<long long>(b) * G + lane) : -1;
     const float u_acc = tok_on ? __ldg(P.u + urow) : 0.f;
     const float u_res = tg_on ? __ldg(P.u + urow + 1) : 0.f;
+    // the two logits at the draft token: left by the sweep CTA of the draft position when the sweep
+    // does that (same round trip), else fetched below (a second one)
+    float2 tl = make_float2(0.f, 0.f);
+    if (P.tokl && tok_on && !greedy) tl = __ldcg(P.tokl + static_cast<long long>(b) * G + lane);
     CtlRegs ctl;
     if ((P.mode & MODE_MLP) && !status) ctl = ctl_load(P, b, lane);
 
-    // ---- second round trip: the two logits at the draft token ----
-    const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb;
-    const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb;
     const bool badtok = tok_on && (x < 0 || x >= P.V);
-    float dxf = 0.f, txf = 0.f;
-    if (tok_on && !badtok && !greedy) {
+    float dxf = tl.x, txf = tl.y;
+    if (!P.tokl && tok_on && !badtok && !greedy) {
+        const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb;
+        const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb;
         dxf = elem_to_float(drow + static_cast<long long>(lane) * P.dsp, x);
         txf = elem_to_float(trow + static_cast<long long>(lane) * P.tsp, x);
     }
@@ -793,36 +825,8 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         if (__any_sync(0xffffffffu, badtok)) status |= 2;
     }
 
-    // signals
-    const float in_bits = P.bits ? static_cast<float>(kLog2e) : 1.f;
-    const float Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.f;
-    const float Cout = (status == 0 && lane < gam) ? ci : 0.f;
-    float f4[4] = {0.f, 0.f, 0.f, 0.f};
-    if (status == 0) {
-        f4[0] = warp_sumf(Hout) / static_cast<float>(gam);
-        f4[1] = warp_sumf(Cout) / static_cast<float>(gam);
-        f4[2] = warp_maxf(Hout);
-        f4[3] = -warp_maxf(lane < gam ? -Cout : -2.f);
-    }
-    if (lane < G) {
-        if (P.H) P.H[static_cast<long long>(b) * G + lane] = Hout;
-        if (P.C) P.C[static_cast<long long>(b) * G + lane] = Cout;
-    }
-    if (P.feat && lane < 4)
-        P.feat[static_cast<long long>(b) * 4 + lane] = lane == 0 ? f4[0] : lane == 1 ? f4[1] : lane == 2 ? f4[2] : f4[3];
-
-    if (P.mode & MODE_MLP) {
-        if (status == 0) {
-            ctl_eval(P, ctl, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr,
-                     P.gamma_next + b);
-        } else {
-            if (P.scores && lane < P.n_out) P.scores[static_cast<long long>(b) * P.n_out + lane] = 0.f;
-            if (lane == 0) P.gamma_next[b] = 0;
-        }
-    }
-
-    // acceptance comes last: the two logits at the draft token had the whole signal and controller
-    // work above to arrive
+    // Acceptance first: the resample kernel waits for this row's stop position, nothing waits for
+    // the signals and the controller, which follow the completion flag.
     if (status == 0 && tok_on) {
         if (greedy) {
             accept = (x == amax);
@@ -864,6 +868,35 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         }
     }
     if (P.status && lane == 0) P.status[b] = status;
+    row_done_signal(P, b);
+
+    // signals
+    const float in_bits = P.bits ? static_cast<float>(kLog2e) : 1.f;
+    const float Hout = (status == 0 && lane < gam) ? Hi * in_bits : 0.f;
+    const float Cout = (status == 0 && lane < gam) ? ci : 0.f;
+    float f4[4] = {0.f, 0.f, 0.f, 0.f};
+    if (status == 0) {
+        f4[0] = warp_sumf(Hout) / static_cast<float>(gam);
+        f4[1] = warp_sumf(Cout) / static_cast<float>(gam);
+        f4[2] = warp_maxf(Hout);
+        f4[3] = -warp_maxf(lane < gam ? -Cout : -2.f);
+    }
+    if (lane < G) {
+        if (P.H) P.H[static_cast<long long>(b) * G + lane] = Hout;
+        if (P.C) P.C[static_cast<long long>(b) * G + lane] = Cout;
+    }
+    if (P.feat && lane < 4)
+        P.feat[static_cast<long long>(b) * 4 + lane] = lane == 0 ? f4[0] : lane == 1 ? f4[1] : lane == 2 ? f4[2] : f4[3];
+
+    if (P.mode & MODE_MLP) {
+        if (status == 0) {
+            ctl_eval(P, ctl, f4, P.scores ? P.scores + static_cast<long long>(b) * P.n_out : nullptr,
+                     P.gamma_next + b);
+        } else {
+            if (P.scores && lane < P.n_out) P.scores[static_cast<long long>(b) * P.n_out + lane] = 0.f;
+            if (lane == 0) P.gamma_next[b] = 0;
+        }
+    }
 }
 
 // Epilogue of the draft-side sampling sweep (one warp per batch row): lane i merges the partials
@@ -909,15 +942,28 @@ __device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, f
     if (P.status && lane == 0) P.status[b] = status;
 }
 
+// One CTA's share of a batch row's fresh-token draw (defined with the resample kernel below).
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void resample_body(const KParams& P, const int bid);
+
 // ----------------------------------------------------------------------------------------
-// Sweep kernel
+// Sweep kernel.  CTAs 0 .. n_sweep-1 sweep one slice of one logit row each.  With verification the
+// grid may carry B*R more CTAs behind them that do the resample kernel's work in the same launch:
+// CTAs start in index order, so these start exactly when the sweep runs out of slices, wait (with
+// a bound) for their batch row's completion flag and fill the SMs that the sweep's last CTAs
+// leave one by one.  A second launch, even a programmatic dependent one, starts microseconds
+// after the last sweep CTA has started and leaves most of the drain unused.
 // ----------------------------------------------------------------------------------------
 template <typename T, bool ALIGNED, int U>
 __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __grid_constant__ KParams P) {
+    if (static_cast<int>(blockIdx.x) >= P.n_sweep) {
+        resample_body<T, ALIGNED>(P, static_cast<int>(blockIdx.x) - P.n_sweep);
+        return;
+    }
     __shared__ float4 sh_part[kWarps];
     __shared__ int sh_count;
     __shared__ float sh_m0[kWarps];
-    asm volatile("griddepcontrol.launch_dependents;");  // the resample kernel may be scheduled as SMs free up
+    asm volatile("griddepcontrol.launch_dependents;");  // a dependent resample kernel may be scheduled as SMs free up
     if (threadIdx.x == 0) sh_count = 0;
     if (threadIdx.x < kWarps) sh_m0[threadIdx.x] = kFloor;
     __syncthreads();  // before any load is issued
@@ -963,6 +1009,16 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
         } else {
             const T* row = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb +
                            static_cast<long long>(pos) * P.dsp;
+            if (verify && P.tokl && s == 0 && threadIdx.x == 0 && !greedy) {
+                // the acceptance test of this position needs both logits at the draft token: fetch them
+                // now, while the sweep hides the latency, and leave them for the row epilogue
+                const int x = __ldg(P.tok + static_cast<long long>(b) * P.G + pos);
+                if (x >= 0 && x < P.V) {
+                    const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
+                                    static_cast<long long>(pos) * P.tsp;
+                    P.tokl[static_cast<long long>(b) * P.G + pos] = make_float2(elem_to_float(row, x), elem_to_float(trow, x));
+                }
+            }
             part = sweep_warp<T, ALIGNED, PATH_DRAFT, U, STEP>(row, lo, hi, first, scale, sh_m0);
             path = PATH_DRAFT;
         }
@@ -985,15 +1041,17 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
             }
             P.part[static_cast<long long>(blockIdx.x)] = acc;
         }
-    } else if (warp != 0) {
-        return;
+    } else if (row_ok || rem != 0 || warp != 0) {
+        return;  // unused position: nothing to count; a flagged row keeps its first CTA for the epilogue
     }
 
-    // ticket: the last CTA of this batch row runs the row epilogue; nobody waits
+    // ticket: the last of the row's active CTAs runs the row epilogue; nobody waits
+    const int n_rows = P.sample ? gam : (verify ? 2 * gam + 1 : gam);
+    const int n_tickets = row_ok ? n_rows * P.nsplit : 1;
     int last_row = 0;
     if (lane == 0) {
         __threadfence();
-        last_row = (atomicAdd(P.tick1 + b, 1) == per_row - 1);
+        last_row = (atomicAdd(P.tick1 + b, 1) == n_tickets - 1);
     }
     if (!__shfl_sync(0xffffffffu, last_row, 0)) return;
     __threadfence();
@@ -1173,23 +1231,42 @@ __device__ __forceinline__ double rs_total(const RsSums& cs, int nchunk, int per
 }
 
 template <typename T, bool ALIGNED>
-__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ KParams P) {
+__device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     __shared__ int sh_flag;
     __shared__ int sh_empty;
     __shared__ float sh_cs[kRsStage];
-    // launched as a programmatic dependent of the sweep kernel: its CTAs may already be resident
-    // while the sweep's last CTAs finish; nothing the sweep wrote is read before this returns
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
-    // (last batch row first: the sweep touched those rows most recently, part of them is still in L2)
     // (draft-side sampling: one draw per drafted position; r counts positions, b = r / gamma_max)
-    const int n_draws = P.sample ? P.B * P.G : P.B;
-    const int bq = blockIdx.x / P.R;
-    const int share = blockIdx.x - bq * P.R;
-    const int r = n_draws - 1 - bq;
+    const int bq = bid / P.R;
+    const int share = bid - bq * P.R;
+    const int r = P.rs_reverse ? (P.sample ? P.B * P.G : P.B) - 1 - bq : bq;
     const int b = P.sample ? r / P.G : r;
-    const RowInfo ri = P.info[r];
+    // Launched as a programmatic dependent of the sweep kernel, so its CTAs become resident as the
+    // sweep's last CTAs leave.  With completion flags a CTA waits only for its own batch row (rows
+    // are taken in the order the sweep finishes them unless rs_reverse is set) and the stop positions of finished rows are
+    // summed while the sweep drains; every sweep CTA is resident or done before the first CTA of
+    // this kernel starts, so the wait ends, and it is bounded all the same.  Without flags the CTA
+    // waits for the whole sweep grid.
+    if (P.rdone) {
+        if (threadIdx.x == 0) sh_flag = row_done_wait(P.rdone + b) ? 1 : 0;
+        __syncthreads();
+        if (!sh_flag) {
+            if (threadIdx.x == 0 && share == 0 && P.status) atomicOr(P.status + b, 16);
+            return;
+        }
+        __syncthreads();  // sh_flag is reused below
+    } else {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    RowInfo ri;
+    {
+        const int4* ip = reinterpret_cast<const int4*>(P.info + r);
+        const int4 lo4 = __ldcg(ip), hi4 = __ldcg(ip + 1);
+        ri.mode = lo4.x; ri.n = lo4.y; ri.u2 = __int_as_float(lo4.z); ri.scale = __int_as_float(lo4.w);
+        ri.lse2_p = __hiloint2double(hi4.y, hi4.x);
+        ri.lse2_q = __hiloint2double(hi4.w, hi4.z);
+    }
     if (ri.mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
     const long long out_at = P.sample ? static_cast<long long>(r) : static_cast<long long>(b) * (P.G + 1) + ri.n;
 
@@ -1300,6 +1377,11 @@ __global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_cons
         int tok = (found != 0x7fffffff) ? found : lastw;
         P.out_tok[out_at] = tok;
     }
+}
+
+template <typename T, bool ALIGNED>
+__global__ void __launch_bounds__(kThreads, 4) resample_kernel(const __grid_constant__ KParams P) {
+    resample_body<T, ALIGNED>(P, static_cast<int>(blockIdx.x));
 }
 
 // ----------------------------------------------------------------------------------------
