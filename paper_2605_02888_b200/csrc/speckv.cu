@@ -49,13 +49,17 @@ int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
     return ns;
 }
 
+#ifndef SPECKV_RS_CHUNKS
+#define SPECKV_RS_CHUNKS 64  // 256-element chunks of the stop position that one resample CTA sums
+#endif
+
 Plan make_plan(const speckv_batch* bt) {
     Plan p;
     const size_t B = static_cast<size_t>(bt->B);
     p.J_full = 2 * bt->gamma_max + 1;
     p.nvec = (bt->V + kVec - 1) / kVec;
     p.nchunk = (bt->V + kChunk - 1) / kChunk;
-    p.R = (p.nchunk + 63) / 64;
+    p.R = (p.nchunk + SPECKV_RS_CHUNKS - 1) / SPECKV_RS_CHUNKS;
     if (p.R > 32) p.R = 32;
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;

@@ -1147,35 +1147,45 @@ __device__ __forceinline__ void rs_chunk_weights(const RsConst& c, const T* trow
     rs_weights<T>(c, rt, rd, w);
 }
 
-// Each warp takes two chunks at a time (c0+warp, +8) and requests the next two before it evaluates
-// the current ones, so the memory latency is paid once per CTA, not once per batch.
-template <typename T, bool ALIGNED>
-__device__ __forceinline__ void rs_load_batch(const RsConst& c, const T* trow, const T* drow, int base, int c1, int V,
-                                              Raw<T> (&rt)[2], Raw<T> (&rd)[2]) {
+// Each warp takes KU chunks at a time (c0+warp, +8, ...) and requests the next KU before it evaluates
+// the current ones, so the memory latency is paid once per CTA, not once per batch.  MODE is the
+// row's mode as a constant: a bonus draw never touches the draft row, so its registers go into a
+// deeper batch instead.  The buffers of both batches stay within 32 registers per thread for
+// either element type; more than that spills and the kernel falls to a fraction of its rate.
+template <typename T, bool ALIGNED, int MODE, int KU>
+__device__ __forceinline__ void rs_load_batch(const T* trow, const T* drow, int base, int c1, int V,
+                                              Raw<T> (&rt)[KU], Raw<T> (&rd)[KU]) {
+    const float ninf = __int_as_float(0xff800000);
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
+    for (int u = 0; u < KU; ++u) {
         const int ch = base + u * kWarps;
-        if (ch < c1) rs_load<T, ALIGNED>(c, trow, drow, ch, V, rt[u], rd[u]);
-        else { rt[u] = raw_fill<T>(__int_as_float(0xff800000)); rd[u] = rt[u]; }
+        const int e0 = ch * kChunk + (threadIdx.x & 31) * kVec;
+        if (ch < c1) {
+            rt[u] = load_raw<T, ALIGNED>(trow, e0, V, ninf);
+            if (MODE == RS_RESIDUAL) rd[u] = load_raw<T, ALIGNED>(drow, e0, V, ninf);
+        } else {
+            rt[u] = raw_fill<T>(ninf);
+            if (MODE == RS_RESIDUAL) rd[u] = rt[u];
+        }
     }
 }
 
-template <typename T, bool ALIGNED>
-__device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
-                                              int V, float* csum) {
-    constexpr int kU = 2;
+template <typename T, bool ALIGNED, int MODE, int KU>
+__device__ __forceinline__ void rs_chunk_sums_mode(RsConst c, const T* trow, const T* drow, int c0, int c1,
+                                                   int V, float* csum) {
+    c.mode = MODE;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int base = c0 + warp;
     if (base >= c1) return;
-    Raw<T> rt[kU], rd[kU];
-    rs_load_batch<T, ALIGNED>(c, trow, drow, base, c1, V, rt, rd);
+    Raw<T> rt[KU], rd[KU];
+    rs_load_batch<T, ALIGNED, MODE, KU>(trow, drow, base, c1, V, rt, rd);
     while (base < c1) {
-        const int next = base + kWarps * kU;
-        Raw<T> nt[kU], nd[kU];
-        if (next < c1) rs_load_batch<T, ALIGNED>(c, trow, drow, next, c1, V, nt, nd);
-        float s[kU];
+        const int next = base + kWarps * KU;
+        Raw<T> nt[KU], nd[KU];
+        if (next < c1) rs_load_batch<T, ALIGNED, MODE, KU>(trow, drow, next, c1, V, nt, nd);
+        float s[KU];
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
+        for (int u = 0; u < KU; ++u) {
             float w[kVec];
             rs_weights<T>(c, rt[u], rd[u], w);
             s[u] = 0.f;
@@ -1185,19 +1195,31 @@ __device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, c
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-            for (int u = 0; u < kU; ++u) s[u] = __fadd_rn(s[u], __shfl_xor_sync(0xffffffffu, s[u], o));
+            for (int u = 0; u < KU; ++u) s[u] = __fadd_rn(s[u], __shfl_xor_sync(0xffffffffu, s[u], o));
         }
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
+        for (int u = 0; u < KU; ++u) {
             const int ch = base + u * kWarps;
             if (lane == 0 && ch < c1) csum[ch] = s[u];
         }
         if (next < c1) {
 #pragma unroll
-            for (int u = 0; u < kU; ++u) { rt[u] = nt[u]; rd[u] = nd[u]; }
+            for (int u = 0; u < KU; ++u) {
+                rt[u] = nt[u];
+                if (MODE == RS_RESIDUAL) rd[u] = nd[u];
+            }
         }
         base = next;
     }
+}
+
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
+                                              int V, float* csum) {
+    constexpr int kResidual = sizeof(T) == 2 ? 2 : 1;  // chunks per batch: two rows to buffer
+    constexpr int kBonus = 2 * kResidual;              // one row to buffer
+    if (c.mode == RS_BONUS) rs_chunk_sums_mode<T, ALIGNED, RS_BONUS, kBonus>(c, trow, drow, c0, c1, V, csum);
+    else rs_chunk_sums_mode<T, ALIGNED, RS_RESIDUAL, kResidual>(c, trow, drow, c0, c1, V, csum);
 }
 
 // The last CTA of a row copies the row's chunk sums into shared memory (one memory round trip for
