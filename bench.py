@@ -4,8 +4,9 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload b256]
 
 A step = one pass of the whole hot path (draft signals, controller, verification: a memset of the
-tickets, the sweep kernel and the resample kernel) over one synthetic batch whose logits are
-resident in HBM.
+tickets, then the sweep kernel, whose grid also draws the fresh tokens for bf16 logits; for fp32
+logits the ring sweep and the resample kernel) over one synthetic batch whose logits are resident
+in HBM.
 Prints ONE JSON line: verified speculation rows/s (whole job), the roofline of the dominant
 kernel against the measured HBM peak, the end-to-end figure with host buffers, and the CPU
 oracle timed on the host cores as a reported baseline.  With --impl reference the oracle
@@ -267,11 +268,17 @@ def main():
     bytes_avg = sum(bytes_step[i % n_batches] for i in range(n_prof)) / n_prof
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_avg / (sweep_avg * 1e-3) / 1e9
-    kernel = "pipe_sweep_kernel" if w.dtype == "fp32" else "sweep_kernel"  # the library picks by logit type
+    # the library picks by logit type: fp32 -> ring sweep, then a resample kernel (two launches per step);
+    # bf16 -> register-staged sweep whose grid also carries the resample CTAs (one launch per step, so
+    # its duration is that of the whole pass over the batch, second read of the stop positions included)
+    kernel = "pipe_sweep_kernel" if w.dtype == "fp32" else "sweep_kernel"
+    one_launch = kernel == "sweep_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,
                 "algorithmic_bytes_per_launch": bytes_avg, "kernel_ms": sweep_avg,
-                "kernel_ms_min": min(sweep_ms), "resample_kernel_ms": sum(resample_ms) / n_prof,
+                "kernel_ms_min": min(sweep_ms),
+                "kernel_covers": "sweep + row epilogues + fresh-token draw" if one_launch else "sweep + row epilogues",
+                "resample_kernel_ms": None if one_launch else sum(resample_ms) / n_prof,
                 "timed_over": f"{n_prof} steps after the timed region, CUDA events recorded inside the library call",
                 "frac_of_8TBps": achieved / 8000.0,
                 "step_GBps": sum(bytes_step[i % n_batches] for i in range(args.steps)) / args.steps / (ms_step * 1e-3) / 1e9}
@@ -352,7 +359,7 @@ def main():
                        "l2": f"{n_batches} resident batches of {bytes_step[0] / 1e6:.0f} MB alternate (each larger than L2)",
                        "parallelism": f"dp{world} (rows sharded, no collective)"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
-            "gpu_launches": 2 * args.steps,
+            "gpu_launches": (1 if one_launch else 2) * args.steps,
             "tokens_per_step_mean": float(outs[0].n_accepted.float().mean()) + 1.0,
         }))
     if dist:

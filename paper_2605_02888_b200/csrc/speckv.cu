@@ -146,6 +146,13 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
 
 // 1: after the register-staged sweep the fresh tokens are drawn by extra CTAs of the same launch;
 // 0: always by a second kernel (measurement builds)
+// the rows swept last have their fresh tokens drawn by more, shorter CTAs (see resample_body)
+#ifndef SPECKV_RS_TAIL_ROWS
+#define SPECKV_RS_TAIL_ROWS 16
+#endif
+#ifndef SPECKV_RS_TAIL_MULT
+#define SPECKV_RS_TAIL_MULT 2
+#endif
 #ifndef SPECKV_MERGED
 #define SPECKV_MERGED 1
 #endif
@@ -155,8 +162,15 @@ cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged
     constexpr int U = sizeof(T) == 2 ? SPECKV_U : (SPECKV_U + 1) / 2;
     const bool verify = (P.mode & MODE_VERIFY) != 0;
     const bool ring = ALIGNED && staged;
-    const long long n_draw = static_cast<long long>(P.B) * P.R;
-    const bool merged = SPECKV_MERGED && verify && !ring && P.rdone && P.n_sweep + n_draw <= 0x7fffffffLL;
+    P.rs_tail = 0; P.R2 = P.R; P.chunks_per_cta2 = P.chunks_per_cta;
+    bool merged = SPECKV_MERGED && verify && !ring && P.rdone;
+    if (merged && P.B >= 4 * SPECKV_RS_TAIL_ROWS && P.R * SPECKV_RS_TAIL_MULT <= 32 && SPECKV_RS_TAIL_MULT > 1) {
+        P.rs_tail = SPECKV_RS_TAIL_ROWS;
+        P.R2 = P.R * SPECKV_RS_TAIL_MULT;
+        P.chunks_per_cta2 = (P.nchunk + P.R2 - 1) / P.R2;
+    }
+    const long long n_draw = static_cast<long long>(P.B - P.rs_tail) * P.R + static_cast<long long>(P.rs_tail) * P.R2;
+    merged = merged && P.n_sweep + n_draw <= 0x7fffffffLL;
     if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
     cudaError_t e;
     if (ring) {

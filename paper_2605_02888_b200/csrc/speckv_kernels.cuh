@@ -53,6 +53,7 @@ struct KParams {
     int B, G, V, J, nsplit, nvec, per_split, nchunk, R, chunks_per_cta, mode, bits;
     int n_sweep;  // sweep kernel: CTAs that sweep; the rest of the grid (if any) does the resample work
     int sample;  // 1: draft-side sampling (every drafted position draws a token from its own row)
+    int rs_tail, R2, chunks_per_cta2;  // resample: the last rs_tail draws in launch order use R2 CTAs each
     int rs_reverse;  // resample kernel: 1 = last batch row first (after a sweep it cannot overlap: those rows are the freshest in L2)
     int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
@@ -1217,7 +1218,7 @@ template <typename T, bool ALIGNED>
 __device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, const T* drow, int c0, int c1,
                                               int V, float* csum) {
     constexpr int kResidual = sizeof(T) == 2 ? 2 : 1;  // chunks per batch: two rows to buffer
-    constexpr int kBonus = 2 * kResidual;              // one row to buffer
+    constexpr int kBonus = 2;  // one row to buffer; measured: deeper bf16 batches leave a warp too few iterations
     if (c.mode == RS_BONUS) rs_chunk_sums_mode<T, ALIGNED, RS_BONUS, kBonus>(c, trow, drow, c0, c1, V, csum);
     else rs_chunk_sums_mode<T, ALIGNED, RS_RESIDUAL, kResidual>(c, trow, drow, c0, c1, V, csum);
 }
@@ -1260,8 +1261,15 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
     // (draft-side sampling: one draw per drafted position; r counts positions, b = r / gamma_max)
-    const int bq = bid / P.R;
-    const int share = bid - bq * P.R;
+    // the last rs_tail draws (in launch order) are cut into R2 >= R shares: their rows are the last to
+    // be swept, nothing is left to overlap their draw with, and more CTAs per row shorten it
+    const int n_all = P.sample ? P.B * P.G : P.B;
+    const int n_head = (n_all - P.rs_tail) * P.R;
+    const bool tail = bid >= n_head;
+    const int Rr = tail ? P.R2 : P.R;
+    const int cpc = tail ? P.chunks_per_cta2 : P.chunks_per_cta;
+    const int bq = tail ? (n_all - P.rs_tail) + (bid - n_head) / Rr : bid / Rr;
+    const int share = tail ? (bid - n_head) % Rr : bid - bq * Rr;
     const int r = P.rs_reverse ? (P.sample ? P.B * P.G : P.B) - 1 - bq : bq;
     const int b = P.sample ? r / P.G : r;
     // Launched as a programmatic dependent of the sweep kernel, so its CTAs become resident as the
@@ -1299,15 +1307,15 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     float* csum = P.csum + static_cast<long long>(r) * P.nchunk;
     RsConst c = rs_const(ri, ri.mode);
 
-    const int c0 = share * P.chunks_per_cta;
-    const int c1 = min(P.nchunk, c0 + P.chunks_per_cta);
+    const int c0 = share * cpc;
+    const int c1 = min(P.nchunk, c0 + cpc);
     rs_chunk_sums<T, ALIGNED>(c, trow, drow, c0, c1, P.V, csum);
 
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
         int old = atomicAdd(P.tick2 + r, 1);
-        sh_flag = (old == P.R - 1);
+        sh_flag = (old == Rr - 1);
     }
     __syncthreads();
     if (!sh_flag) return;
