@@ -28,8 +28,8 @@
  *   - The return code covers what the host can check (NULL or inconsistent arguments,
  *     unsupported sizes, workspace too small, launch failure).  Data-dependent problems are
  *     reported per row in row_status[b]; such a row gets n_accepted = 0, out_tokens = -1,
- *     gamma_next = 0 and zeros in its float outputs.  No kernel traps; the only waits (inside
- *     the sweep used for fp32 logits) are bounded and end in SPECKV_ROW_TIMEOUT on the row at hand.
+ *     gamma_next = 0 and zeros in its float outputs.  No kernel traps; every wait inside a
+ *     kernel is bounded and ends in SPECKV_ROW_TIMEOUT on the row at hand.
  *   - Logits below -2^100 are treated as -inf (probability 0).  NaN or +inf anywhere in a used
  *     logit row, or a used row without any finite entry, flags the row.
  *   - Temperature: 0 selects the greedy rule (and T = 1 for that row's signals); otherwise
@@ -63,7 +63,7 @@ enum {
     SPECKV_ROW_BAD_TOKEN = 2,       /* a used draft token outside 0..V-1                  */
     SPECKV_ROW_NONFINITE = 4,       /* NaN / +inf / all -inf in a used logit row          */
     SPECKV_ROW_BAD_TEMPERATURE = 8, /* negative, NaN or infinite temperature              */
-    SPECKV_ROW_TIMEOUT = 16         /* a bounded wait inside the ring sweep ran out        */
+    SPECKV_ROW_TIMEOUT = 16         /* a bounded wait inside a kernel ran out              */
 };
 
 #define SPECKV_MAX_GAMMA 16  /* gamma_max <= 16                                           */
