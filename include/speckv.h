@@ -151,9 +151,10 @@ speckv_status speckv_step(const speckv_batch* batch, const float* comp, const sp
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Measurement aid: speckv_step with three caller-created CUDA events (cudaEvent_t passed as
- * void*) recorded on the stream before the sweep kernel, between the sweep and the resample
- * kernel, and after the resample kernel, so that a benchmark can time the dominant kernel
- * alone.  Results are identical to speckv_step.  Any event may be NULL.                   */
+ * void*) recorded on the stream before the sweep kernel, after it, and after the resample
+ * kernel, so that a benchmark can time the dominant kernel alone.  Where the sweep kernel's own
+ * grid draws the fresh tokens (bf16 logits) there is no resample kernel and the last two events
+ * coincide.  Results are identical to speckv_step.  Any event may be NULL.                 */
 speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
                                    float* H, float* C, float* feat, float* scores,
                                    int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens,
@@ -187,6 +188,45 @@ speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp,
 #define SPECKV_STATIC_SCRATCH_BYTES (4u << 20)
 speckv_status speckv_signals_static(const speckv_batch* batch, float* H, float* C, float* feat,
                                     int32_t* row_status, void* cuda_stream);
+
+/* ---- Vocabulary-sharded step (the verification of Sec. 3.1 and the signals of Sec. 4.1 when the
+ * vocabulary axis of the logits is split over n_shards devices, as a tensor-parallel output
+ * projection leaves them).  Shard r holds columns [v_begin_r, v_begin_r + V_r) of every logit row:
+ * `local` is an ordinary speckv_batch whose V is V_r and whose logit pointers and strides describe
+ * the local slice; draft_tokens, gamma, temperature and uniforms are the full batch's, identical
+ * on every shard.  All shards but the last have the same width (shard_width); the last may be
+ * narrower.  The results equal those of speckv_step on the concatenated logits (same tolerance,
+ * same near-tie caveats).  The four calls run on every shard, in this order, with two small
+ * exchanges and one reduction between them that the caller performs (any all-gather will do):
+ *
+ *   speckv_shard_sweep      local slice -> shard_state [B, 2*gamma_max+1, 4] fp32, shard_tokl [B, gamma_max, 2] fp32
+ *      -- all-gather both over the shards, in shard order: all_state [n_shards, B, 2*gamma_max+1, 4],
+ *         all_tokl [n_shards, B, gamma_max, 2]
+ *   speckv_shard_finish     every output of speckv_step except the fresh token of sampled rows (its
+ *                           slot holds -1), and row_info (SPECKV_ROW_INFO_BYTES per row, opaque,
+ *                           16-byte aligned) for the next two calls; identical on every shard
+ *   speckv_shard_draw_sums  local slice -> shard_weight [B, 2] fp64
+ *      -- all-gather: all_weight [n_shards, B, 2]
+ *   speckv_shard_draw_pick  the shard that holds the drawn token writes it into out_tokens[b, n_accepted[b]]
+ *      -- element-wise maximum of out_tokens over the shards.
+ *
+ * The workspace (speckv_shard_workspace_size(local) bytes, 256-byte aligned) is the shard's own;
+ * its contents must survive from speckv_shard_draw_sums to speckv_shard_draw_pick.  All pointers are
+ * device pointers; n_shards <= 32.  mlp may be NULL (no controller: scores and gamma_next untouched). */
+#define SPECKV_ROW_INFO_BYTES 32
+speckv_status speckv_shard_workspace_size(const speckv_batch* local, size_t* bytes);
+speckv_status speckv_shard_sweep(const speckv_batch* local, int64_t v_begin, float* shard_state, float* shard_tokl,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+speckv_status speckv_shard_finish(const speckv_batch* local, int32_t n_shards, int32_t shard_width, int32_t V_total,
+                                  const float* all_state, const float* all_tokl, const float* comp,
+                                  const speckv_mlp* mlp, float* H, float* C, float* feat, float* scores,
+                                  int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status,
+                                  void* row_info, void* cuda_stream);
+speckv_status speckv_shard_draw_sums(const speckv_batch* local, const void* row_info, double* shard_weight,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+speckv_status speckv_shard_draw_pick(const speckv_batch* local, int64_t v_begin, int32_t rank, int32_t n_shards,
+                                     const void* row_info, const double* all_weight, int32_t* out_tokens,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 const char* speckv_status_string(speckv_status s);
 int speckv_version(void);

@@ -84,6 +84,17 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_step.argtypes = [C.POINTER(_CBatch), vp, C.POINTER(_CMlp)] + [vp] * 8 + [vp, sz, vp]
     L.speckv_step_profiled.restype = C.c_int
     L.speckv_step_profiled.argtypes = L.speckv_step.argtypes + [vp, vp, vp]
+    i32, i64 = C.c_int32, C.c_int64
+    L.speckv_shard_workspace_size.restype = C.c_int
+    L.speckv_shard_workspace_size.argtypes = [C.POINTER(_CBatch), C.POINTER(sz)]
+    L.speckv_shard_sweep.restype = C.c_int
+    L.speckv_shard_sweep.argtypes = [C.POINTER(_CBatch), i64, vp, vp, vp, sz, vp]
+    L.speckv_shard_finish.restype = C.c_int
+    L.speckv_shard_finish.argtypes = [C.POINTER(_CBatch), i32, i32, i32, vp, vp, vp, C.POINTER(_CMlp)] + [vp] * 8 + [vp, vp]
+    L.speckv_shard_draw_sums.restype = C.c_int
+    L.speckv_shard_draw_sums.argtypes = [C.POINTER(_CBatch), vp, vp, vp, sz, vp]
+    L.speckv_shard_draw_pick.restype = C.c_int
+    L.speckv_shard_draw_pick.argtypes = [C.POINTER(_CBatch), i64, i32, i32, vp, vp, vp, vp, sz, vp]
     L.speckv_status_string.restype = C.c_char_p
     L.speckv_status_string.argtypes = [C.c_int]
     L.speckv_version.restype = C.c_int
@@ -381,3 +392,78 @@ def speckv_step(batch: Batch, comp: Optional[torch.Tensor], mlp: Mlp, out: Optio
     if rc != OK:
         raise SpeckvError(rc, "speckv_step")
     return o.as_dict()
+
+
+# ---- vocabulary-sharded step: the four calls of include/speckv.h, argument marshalling only ----
+ROW_INFO_BYTES = 32
+
+
+def shard_workspace(local: Batch) -> torch.Tensor:
+    L = load_library()
+    c = local._c()
+    n = C.c_size_t(0)
+    rc = L.speckv_shard_workspace_size(C.byref(c), C.byref(n))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_shard_workspace_size")
+    return torch.empty(max(int(n.value), 256), dtype=torch.uint8, device=local.draft_logits.device)
+
+
+def speckv_shard_sweep(local: Batch, v_begin: int, shard_state: torch.Tensor, shard_tokl: torch.Tensor,
+                       workspace: torch.Tensor):
+    """Local slice -> shard_state [B, 2G+1, 4] fp32, shard_tokl [B, G, 2] fp32 (both written)."""
+    L = load_library()
+    c = local._c()
+    dev = local.draft_logits.device
+    with torch.cuda.device(dev):
+        rc = L.speckv_shard_sweep(C.byref(c), int(v_begin), _dev_ptr(shard_state, torch.float32, "shard_state"),
+                                  _dev_ptr(shard_tokl, torch.float32, "shard_tokl"), _ptr(workspace),
+                                  workspace.numel(), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_shard_sweep")
+
+
+def speckv_shard_finish(local: Batch, n_shards: int, shard_width: int, V_total: int, all_state: torch.Tensor,
+                        all_tokl: torch.Tensor, comp: Optional[torch.Tensor], mlp: Optional[Mlp], out: "StepOutputs",
+                        row_info: torch.Tensor):
+    """Gathered states -> every step output but the sampled rows' fresh token; row_info for the draw."""
+    L = load_library()
+    c = local._c()
+    m = mlp._c() if mlp is not None else None
+    dev = local.draft_logits.device
+    with torch.cuda.device(dev):
+        rc = L.speckv_shard_finish(C.byref(c), n_shards, shard_width, V_total,
+                                   _dev_ptr(all_state, torch.float32, "all_state"),
+                                   _dev_ptr(all_tokl, torch.float32, "all_tokl"),
+                                   _dev_ptr(comp, torch.float32, "comp"), C.byref(m) if m is not None else None,
+                                   _ptr(out.H), _ptr(out.C), _ptr(out.feat), _ptr(out.scores), _ptr(out.gamma_next),
+                                   _ptr(out.n_accepted), _ptr(out.out_tokens), _ptr(out.row_status),
+                                   _ptr(row_info), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_shard_finish")
+
+
+def speckv_shard_draw_sums(local: Batch, row_info: torch.Tensor, shard_weight: torch.Tensor, workspace: torch.Tensor):
+    """Local slice -> shard_weight [B, 2] fp64 (residual mass, target mass of the stop position)."""
+    L = load_library()
+    c = local._c()
+    dev = local.draft_logits.device
+    with torch.cuda.device(dev):
+        rc = L.speckv_shard_draw_sums(C.byref(c), _ptr(row_info), _dev_ptr(shard_weight, torch.float64, "shard_weight"),
+                                      _ptr(workspace), workspace.numel(), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_shard_draw_sums")
+
+
+def speckv_shard_draw_pick(local: Batch, v_begin: int, rank: int, n_shards: int, row_info: torch.Tensor,
+                           all_weight: torch.Tensor, out_tokens: torch.Tensor, workspace: torch.Tensor):
+    """The shard holding the drawn token writes it into out_tokens[b, n_accepted[b]]."""
+    L = load_library()
+    c = local._c()
+    dev = local.draft_logits.device
+    with torch.cuda.device(dev):
+        rc = L.speckv_shard_draw_pick(C.byref(c), int(v_begin), rank, n_shards, _ptr(row_info),
+                                      _dev_ptr(all_weight, torch.float64, "all_weight"),
+                                      _dev_ptr(out_tokens, torch.int32, "out_tokens"), _ptr(workspace),
+                                      workspace.numel(), _stream(dev))
+    if rc != OK:
+        raise SpeckvError(rc, "speckv_shard_draw_pick")

@@ -9,6 +9,7 @@
 
 #include "speckv_kernels.cuh"
 #include "speckv_pipeline.cuh"
+#include "speckv_shard.cuh"
 
 namespace {
 
@@ -377,6 +378,58 @@ cudaError_t static_scratch_address(void** out) {
     return cudaSuccess;
 }
 
+// ---- vocabulary-sharded verification (speckv_shard.cuh) ----
+struct ShardPlan {
+    int nvec, nchunk, R, chunks_per_cta;
+    size_t off_tick, off_part, off_csum, off_csum2, total;
+};
+ShardPlan make_shard_plan(const speckv_batch* bt) {
+    ShardPlan p;
+    const size_t B = static_cast<size_t>(bt->B), J = 2 * static_cast<size_t>(bt->gamma_max) + 1;
+    p.nvec = (bt->V + kVec - 1) / kVec;
+    p.nchunk = (bt->V + kChunk - 1) / kChunk;
+    p.R = (p.nchunk + SPECKV_RS_CHUNKS - 1) / SPECKV_RS_CHUNKS;
+    if (p.R > 32) p.R = 32;
+    if (p.R < 1) p.R = 1;
+    p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
+    size_t off = 0;
+    p.off_tick = off; off = align_up(off + 2 * B * sizeof(int));  // sweep tickets, draw tickets
+    p.off_part = off; off = align_up(off + B * J * kMaxSplit * sizeof(float4));
+    p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
+    p.off_csum2 = off; off = align_up(off + B * p.nchunk * sizeof(float));
+    p.total = off < kAlign ? kAlign : off;
+    return p;
+}
+
+// what every shard call needs from the local batch
+speckv_status shard_params(const speckv_batch* bt, void* ws, size_t ws_bytes, KParams& P, ShardPlan& pl) {
+    speckv_status st = check_batch(bt, true);
+    if (st != SPECKV_OK) return st;
+    pl = make_shard_plan(bt);
+    if (bt->B == 0) return SPECKV_OK;
+    if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SPECKV_ERR_INVALID_ARG;
+    if (ws_bytes < pl.total) return SPECKV_ERR_WORKSPACE;
+    P.B = bt->B; P.G = bt->gamma_max; P.V = bt->V; P.J = 2 * bt->gamma_max + 1;
+    P.nvec = pl.nvec; P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
+    P.mode = MODE_VERIFY; P.bits = bt->entropy_in_bits ? 1 : 0;
+    P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
+    P.t = bt->target_logits; P.tsb = bt->target_stride_b; P.tsp = bt->target_stride_pos;
+    P.tok = bt->draft_tokens; P.gamma = bt->gamma; P.temp = bt->temperature;
+    P.temp_scalar = bt->temperature_scalar; P.u = bt->uniforms;
+    char* w = static_cast<char*>(ws);
+    P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
+    P.tick2 = P.tick1 + P.B;
+    P.part = reinterpret_cast<float4*>(w + pl.off_part);
+    P.csum = reinterpret_cast<float*>(w + pl.off_csum);
+    P.csum2 = reinterpret_cast<float*>(w + pl.off_csum2);
+    return SPECKV_OK;
+}
+bool shard_aligned(const speckv_batch* bt) {
+    const int es = esize(bt->dtype);
+    return rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es) &&
+           rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
+}
+
 }  // namespace
 
 extern "C" {
@@ -469,6 +522,138 @@ speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp,
     ev.after_resample = static_cast<cudaEvent_t>(ev_after_resample);
     return run(batch, MODE_SIGNALS | MODE_VERIFY | MODE_MLP, comp, mlp, H, C, feat, scores, gamma_next,
                n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream, ev);
+}
+
+speckv_status speckv_shard_workspace_size(const speckv_batch* local, size_t* bytes) {
+    if (!bytes) return SPECKV_ERR_INVALID_ARG;
+    if (!local || local->B < 0 || local->gamma_max < 1 || local->V < 1) return SPECKV_ERR_INVALID_ARG;
+    if (local->gamma_max > SPECKV_MAX_GAMMA || local->V > (1 << 30) || local->B > (1 << 24))
+        return SPECKV_ERR_UNSUPPORTED;
+    *bytes = make_shard_plan(local).total;
+    return SPECKV_OK;
+}
+
+speckv_status speckv_shard_sweep(const speckv_batch* local, int64_t v_begin, float* shard_state, float* shard_tokl,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    KParams P{};
+    ShardPlan pl;
+    speckv_status st = shard_params(local, workspace, workspace_bytes, P, pl);
+    if (st != SPECKV_OK || local->B == 0) return st;
+    if (!shard_state || !shard_tokl || v_begin < 0 || v_begin > (1LL << 30)) return SPECKV_ERR_INVALID_ARG;
+    P.nsplit = choose_nsplit(P.B, P.J, P.V, local->dtype);
+    P.per_split = (P.nvec + P.nsplit - 1) / P.nsplit;
+    if (static_cast<long long>(P.B) * P.J * P.nsplit > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+    P.n_sweep = P.B * P.J * P.nsplit;
+    P.v_begin = static_cast<int>(v_begin);
+    P.export_state = 1;
+    P.state = reinterpret_cast<float4*>(shard_state);
+    P.tokl = reinterpret_cast<float2*>(shard_tokl);
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(P.tick1, 0, static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+    if (cudaMemsetAsync(shard_tokl, 0, static_cast<size_t>(P.B) * P.G * sizeof(float2), cs) != cudaSuccess)
+        return SPECKV_ERR_CUDA;
+    const unsigned grid = static_cast<unsigned>(P.n_sweep);
+    constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
+    const bool al = shard_aligned(local);
+    if (local->dtype == SPECKV_BF16) {
+        if (al) sweep_kernel<__nv_bfloat16, true, Ub><<<grid, kThreads, 0, cs>>>(P);
+        else sweep_kernel<__nv_bfloat16, false, Ub><<<grid, kThreads, 0, cs>>>(P);
+    } else {
+        if (al) sweep_kernel<float, true, Uf><<<grid, kThreads, 0, cs>>>(P);
+        else sweep_kernel<float, false, Uf><<<grid, kThreads, 0, cs>>>(P);
+    }
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
+speckv_status speckv_shard_finish(const speckv_batch* local, int32_t n_shards, int32_t shard_width, int32_t V_total,
+                                  const float* all_state, const float* all_tokl, const float* comp,
+                                  const speckv_mlp* mlp, float* H, float* C, float* feat, float* scores,
+                                  int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status,
+                                  void* row_info, void* cuda_stream) {
+    speckv_status st = check_batch(local, true);
+    if (st != SPECKV_OK) return st;
+    if (n_shards < 1 || n_shards > 32 || shard_width < 1 || V_total < 1) return SPECKV_ERR_INVALID_ARG;
+    if (static_cast<long long>(shard_width) * (n_shards - 1) >= V_total) return SPECKV_ERR_INVALID_ARG;
+    if (local->B == 0) return SPECKV_OK;
+    if (!all_state || !all_tokl || !n_accepted || !out_tokens || !row_info) return SPECKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(row_info) % 16 != 0 || reinterpret_cast<uintptr_t>(all_state) % 16 != 0 ||
+        reinterpret_cast<uintptr_t>(all_tokl) % 8 != 0)
+        return SPECKV_ERR_INVALID_ARG;
+    KParams P{};
+    P.B = local->B; P.G = local->gamma_max; P.V = V_total; P.J = 2 * local->gamma_max + 1;
+    P.mode = MODE_SIGNALS | MODE_VERIFY; P.bits = local->entropy_in_bits ? 1 : 0;
+    if (mlp) {
+        st = check_mlp(mlp);
+        if (st != SPECKV_OK) return st;
+        if (!gamma_next || !feat) return SPECKV_ERR_INVALID_ARG;
+        P.mode |= MODE_MLP;
+        fill_mlp(P, mlp, comp);
+    }
+    P.tok = local->draft_tokens; P.gamma = local->gamma; P.temp = local->temperature;
+    P.temp_scalar = local->temperature_scalar; P.u = local->uniforms;
+    P.H = H; P.C = C; P.feat = feat; P.scores = scores; P.gamma_next = gamma_next;
+    P.n_acc = n_accepted; P.out_tok = out_tokens; P.status = row_status;
+    P.part = const_cast<float4*>(reinterpret_cast<const float4*>(all_state));
+    P.part_stride = P.B * P.J;
+    P.n_shards = n_shards; P.shard_width = shard_width;
+    P.tokl = const_cast<float2*>(reinterpret_cast<const float2*>(all_tokl));
+    P.tokl_stride = static_cast<long long>(P.B) * P.G;
+    P.info = static_cast<RowInfo*>(row_info);
+    if (static_cast<long long>(P.B) * P.J > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+    const unsigned grid = static_cast<unsigned>((P.B + kWarps - 1) / kWarps);
+    shard_finish_kernel<float><<<grid, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
+speckv_status speckv_shard_draw_sums(const speckv_batch* local, const void* row_info, double* shard_weight,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    KParams P{};
+    ShardPlan pl;
+    speckv_status st = shard_params(local, workspace, workspace_bytes, P, pl);
+    if (st != SPECKV_OK || local->B == 0) return st;
+    if (!row_info || !shard_weight) return SPECKV_ERR_INVALID_ARG;
+    P.info = static_cast<RowInfo*>(const_cast<void*>(row_info));
+    P.weight = shard_weight;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(P.tick2, 0, static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+    if (static_cast<long long>(P.B) * P.R > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
+    const unsigned grid = static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R);
+    const bool al = shard_aligned(local);
+    if (local->dtype == SPECKV_BF16) {
+        if (al) shard_sums_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, cs>>>(P);
+        else shard_sums_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, cs>>>(P);
+    } else {
+        if (al) shard_sums_kernel<float, true><<<grid, kThreads, 0, cs>>>(P);
+        else shard_sums_kernel<float, false><<<grid, kThreads, 0, cs>>>(P);
+    }
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+}
+
+speckv_status speckv_shard_draw_pick(const speckv_batch* local, int64_t v_begin, int32_t rank, int32_t n_shards,
+                                     const void* row_info, const double* all_weight, int32_t* out_tokens,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    KParams P{};
+    ShardPlan pl;
+    speckv_status st = shard_params(local, workspace, workspace_bytes, P, pl);
+    if (st != SPECKV_OK || local->B == 0) return st;
+    if (!row_info || !all_weight || !out_tokens) return SPECKV_ERR_INVALID_ARG;
+    if (n_shards < 1 || n_shards > 32 || rank < 0 || rank >= n_shards || v_begin < 0 || v_begin > (1LL << 30))
+        return SPECKV_ERR_INVALID_ARG;
+    P.info = static_cast<RowInfo*>(const_cast<void*>(row_info));
+    P.all_weight = all_weight;
+    P.out_tok = out_tokens;
+    P.rank = rank; P.n_shards = n_shards; P.v_begin = static_cast<int>(v_begin);
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    const unsigned grid = static_cast<unsigned>(P.B);
+    const bool al = shard_aligned(local);
+    if (local->dtype == SPECKV_BF16) {
+        if (al) shard_pick_kernel<__nv_bfloat16, true><<<grid, kThreads, 0, cs>>>(P);
+        else shard_pick_kernel<__nv_bfloat16, false><<<grid, kThreads, 0, cs>>>(P);
+    } else {
+        if (al) shard_pick_kernel<float, true><<<grid, kThreads, 0, cs>>>(P);
+        else shard_pick_kernel<float, false><<<grid, kThreads, 0, cs>>>(P);
+    }
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 
 const char* speckv_status_string(speckv_status s) {

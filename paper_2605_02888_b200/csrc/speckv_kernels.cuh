@@ -74,6 +74,18 @@ struct KParams {
     RowInfo* info;
     float4* part;
     float* csum;
+    // vocabulary-sharded verification (speckv_shard.cuh); all zero otherwise
+    int part_stride;   // row epilogue: float4s between successive partials of one logit row (0 = adjacent)
+    int n_shards;      // row epilogue: tokl holds one [B, G] table per shard, tokl_stride float2s apart
+    int shard_width;   //   and the shard owning token x is min(x / shard_width, n_shards - 1)
+    long long tokl_stride;
+    int v_begin;       // sweep: first vocabulary index of this shard's slice (the batch's V is the slice width)
+    int export_state;  // sweep: 1 = the row's last CTA writes the merged per-logit-row states instead of the row epilogue
+    float4* state;     // [B, J] merged states of this shard (export)
+    float* csum2;      // shard draw: chunk sums of p beside the residual's
+    double* weight;    // shard draw: [B, 2] (residual mass, p mass) of this shard
+    const double* all_weight;  // [n_shards, B, 2]
+    int rank;
 };
 
 // ----------------------------------------------------------------------------------------
@@ -756,11 +768,12 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     const bool tok_on = !status && verify && lane < gam;
 
     // ---- first round trip ----
+    const long long ps = P.part_stride > 0 ? P.part_stride : 1;  // partials of a logit row: adjacent, or one per shard
     float4 qd[kPre], qt[kPre];
 #pragma unroll
     for (int k = 0; k < kPre; ++k) {
-        qd[k] = (dr_on && k < nd) ? ldcg4(pd + k) : make_float4(0.f, 0.f, 0.f, 0.f);
-        qt[k] = (tg_on && k < nt) ? ldcg4(pt + k) : make_float4(0.f, 0.f, 0.f, 0.f);
+        qd[k] = (dr_on && k < nd) ? ldcg4(pd + k * ps) : make_float4(0.f, 0.f, 0.f, 0.f);
+        qt[k] = (tg_on && k < nt) ? ldcg4(pt + k * ps) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     const long long urow = (static_cast<long long>(b) * (G + 1) + lane) * 2;
     const int x = tok_on ? __ldg(P.tok + static_cast<long long>(b) * G + lane) : -1;
@@ -769,7 +782,12 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     // the two logits at the draft token: left by the sweep CTA of the draft position when the sweep
     // does that (same round trip), else fetched below (a second one)
     float2 tl = make_float2(0.f, 0.f);
-    if (P.tokl && tok_on && !greedy) tl = __ldcg(P.tokl + static_cast<long long>(b) * G + lane);
+    if (P.tokl && tok_on && !greedy) {
+        long long at = static_cast<long long>(b) * G + lane;
+        if (P.shard_width > 0)  // the table of the shard whose slice holds the token (one more dependent load)
+            at += (x > 0 ? min(x / P.shard_width, P.n_shards - 1) : 0) * P.tokl_stride;
+        tl = __ldcg(P.tokl + at);
+    }
     CtlRegs ctl;
     if ((P.mode & MODE_MLP) && !status) ctl = ctl_load(P, b, lane);
 
@@ -797,8 +815,8 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             if (k < nd) ad = merge_draft(ad, qd[k], scale);
             if (k < nt) at = greedy ? merge_argmax(at, qt[k]) : merge_target(at, qt[k]);
         }
-        for (int k = kPre; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
-        for (int k = kPre; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
+        for (int k = kPre; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k * ps), scale);
+        for (int k = kPre; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k * ps)) : merge_target(at, ldcg4(pt + k * ps));
         if (dr_on) {
             const float m = ad.x, cnt = ad.y, Zx = ad.z, S = ad.w;
             const float Z = cnt + Zx;
@@ -943,6 +961,39 @@ __device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, f
     if (P.status && lane == 0) P.status[b] = status;
 }
 
+// Epilogue of a vocabulary shard's sweep (one warp per batch row): lane i merges this shard's partials
+// of draft position i and of target position i and writes the two merged states; the row epilogue
+// proper runs later on the states of all shards.  An argmax index becomes a global vocabulary index.
+__device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd,
+                                             const float4* pt, int n) {
+    const int lane = threadIdx.x & 31;
+    const int G = P.G;
+    const bool ok = (gam >= 1 && gam <= G) && (Tf >= 0.f) && (Tf != __int_as_float(0x7f800000));
+    const bool greedy = (Tf == 0.f);
+    const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
+    float4* out = P.state + static_cast<long long>(b) * P.J;
+    if (lane < G) {
+        float4 ad = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ok && lane < gam) {
+            ad = ldcg4(pd);
+            for (int k = 1; k < n; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
+        }
+        out[G + 1 + lane] = ad;
+    }
+    if (lane <= G) {
+        float4 at = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (ok && lane <= gam) {
+            at = ldcg4(pt);
+            for (int k = 1; k < n; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
+            if (greedy) {
+                const int idx = __float_as_int(at.y);
+                if (idx != 0x7fffffff) at.y = __int_as_float(idx + P.v_begin);
+            }
+        }
+        out[lane] = at;
+    }
+}
+
 // One CTA's share of a batch row's fresh-token draw (defined with the resample kernel below).
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ void resample_body(const KParams& P, const int bid);
@@ -1013,7 +1064,7 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
             if (verify && P.tokl && s == 0 && threadIdx.x == 0 && !greedy) {
                 // the acceptance test of this position needs both logits at the draft token: fetch them
                 // now, while the sweep hides the latency, and leave them for the row epilogue
-                const int x = __ldg(P.tok + static_cast<long long>(b) * P.G + pos);
+                const int x = __ldg(P.tok + static_cast<long long>(b) * P.G + pos) - P.v_begin;  // index in this slice
                 if (x >= 0 && x < P.V) {
                     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
                                     static_cast<long long>(pos) * P.tsp;
@@ -1059,6 +1110,10 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
     const long long row0 = static_cast<long long>(b) * P.J;
     if (P.sample) {
         sample_epilogue(P, b, gam, Tf, P.part + (row0 + lane) * P.nsplit, P.nsplit);
+        return;
+    }
+    if (P.export_state) {
+        export_epilogue(P, b, gam, Tf, P.part + (row0 + P.G + 1 + lane) * P.nsplit, P.part + (row0 + lane) * P.nsplit, P.nsplit);
         return;
     }
     row_epilogue<T>(P, b, gam, Tf, P.part + (row0 + (verify ? P.G + 1 + lane : lane)) * P.nsplit, P.nsplit,
@@ -1253,6 +1308,74 @@ __device__ __forceinline__ double rs_total(const RsSums& cs, int nchunk, int per
     return warp_sum(own);
 }
 
+// Warp 0 of the CTA that holds a row's chunk sums: the vocabulary index at which the running sum of the
+// weights first exceeds tau (the last index with weight if rounding leaves tau at or above the total).
+// own = this lane's share of the chunk sums as rs_total left it.  The located chunk's weights are
+// recomputed, bit-identical to the first pass.  Every lane returns the index.
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ int rs_search(const RsConst& c, const T* trow, const T* drow, const RsSums& cs, int nchunk,
+                                         int V, double tau, double own, int per_lane) {
+    const int lane = threadIdx.x & 31;
+    // inclusive scan of the per-lane group sums
+    double incl = own;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    unsigned hit = __ballot_sync(0xffffffffu, incl > tau && own > 0.0);
+    unsigned pos = __ballot_sync(0xffffffffu, own > 0.0);
+    int src = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));  // fallback: last group with weight
+    // the chosen lane walks its chunks
+    int chunk = -1;
+    double before = 0.0;
+    if (lane == src) {
+        double run = incl - own;
+        const int a = lane * per_lane, e = min(nchunk, a + per_lane);
+        int last_pos = -1;
+        double last_before = 0.0;
+        for (int ch = a; ch < e; ++ch) {
+            double sv = static_cast<double>(cs[ch]);
+            if (sv > 0.0) { last_pos = ch; last_before = run; }
+            if (run + sv > tau && sv > 0.0) { chunk = ch; before = run; break; }
+            run += sv;
+        }
+        if (chunk < 0) { chunk = last_pos; before = last_before; }
+    }
+    chunk = __shfl_sync(0xffffffffu, chunk, src);
+    before = __shfl_sync(0xffffffffu, before, src);
+
+    // recompute the chunk's weights (bit-identical to the first pass) and scan them
+    float w[kVec];
+    rs_chunk_weights<T, ALIGNED>(c, trow, drow, chunk, V, w);
+    double lane_tot = 0.0;
+#pragma unroll
+    for (int j = 0; j < kVec; ++j) lane_tot += static_cast<double>(w[j]);
+    double lincl = lane_tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        double v = __shfl_up_sync(0xffffffffu, lincl, o);
+        if (lane >= o) lincl += v;
+    }
+    double run = before + (lincl - lane_tot);
+    int found = 0x7fffffff, lastw = -1;
+#pragma unroll
+    for (int j = 0; j < kVec; ++j) {
+        run += static_cast<double>(w[j]);
+        const int idx = chunk * kChunk + lane * kVec + j;
+        if (w[j] > 0.f) {
+            lastw = idx;
+            if (run > tau && found == 0x7fffffff) found = idx;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
+        lastw = max(lastw, __shfl_xor_sync(0xffffffffu, lastw, o));
+    }
+    return (found != 0x7fffffff) ? found : lastw;
+}
+
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     __shared__ int sh_flag;
@@ -1346,67 +1469,8 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     if (warp != 0) return;
 
     const double tau = static_cast<double>(ri.u2) * W;
-    // inclusive scan of the per-lane group sums
-    double incl = own;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        double v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    unsigned hit = __ballot_sync(0xffffffffu, incl > tau && own > 0.0);
-    unsigned pos = __ballot_sync(0xffffffffu, own > 0.0);
-    int src = hit ? (__ffs(hit) - 1) : (31 - __clz(pos));  // fallback: last group with weight
-    // the chosen lane walks its chunks
-    int chunk = -1;
-    double before = 0.0;
-    if (lane == src) {
-        double run = incl - own;
-        const int a = lane * per_lane, e = min(P.nchunk, a + per_lane);
-        int last_pos = -1;
-        double last_before = 0.0;
-        for (int ch = a; ch < e; ++ch) {
-            double sv = static_cast<double>(cs[ch]);
-            if (sv > 0.0) { last_pos = ch; last_before = run; }
-            if (run + sv > tau && sv > 0.0) { chunk = ch; before = run; break; }
-            run += sv;
-        }
-        if (chunk < 0) { chunk = last_pos; before = last_before; }
-    }
-    chunk = __shfl_sync(0xffffffffu, chunk, src);
-    before = __shfl_sync(0xffffffffu, before, src);
-
-    // recompute the chunk's weights (bit-identical to the first pass) and scan them
-    float w[kVec];
-    rs_chunk_weights<T, ALIGNED>(c, trow, drow, chunk, P.V, w);
-    double lane_tot = 0.0;
-#pragma unroll
-    for (int j = 0; j < kVec; ++j) lane_tot += static_cast<double>(w[j]);
-    double lincl = lane_tot;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        double v = __shfl_up_sync(0xffffffffu, lincl, o);
-        if (lane >= o) lincl += v;
-    }
-    double run = before + (lincl - lane_tot);
-    int found = 0x7fffffff, lastw = -1;
-#pragma unroll
-    for (int j = 0; j < kVec; ++j) {
-        run += static_cast<double>(w[j]);
-        const int idx = chunk * kChunk + lane * kVec + j;
-        if (w[j] > 0.f) {
-            lastw = idx;
-            if (run > tau && found == 0x7fffffff) found = idx;
-        }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        found = min(found, __shfl_xor_sync(0xffffffffu, found, o));
-        lastw = max(lastw, __shfl_xor_sync(0xffffffffu, lastw, o));
-    }
-    if (lane == 0) {
-        int tok = (found != 0x7fffffff) ? found : lastw;
-        P.out_tok[out_at] = tok;
-    }
+    const int tok = rs_search<T, ALIGNED>(c, trow, drow, cs, P.nchunk, P.V, tau, own, per_lane);
+    if (lane == 0) P.out_tok[out_at] = tok;
 }
 
 template <typename T, bool ALIGNED>

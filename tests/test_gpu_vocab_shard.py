@@ -1,0 +1,83 @@
+"""Vocabulary-sharded step against the CPU oracle on the concatenated logits: the shards' calls run
+one after the other on one device (no kernel waits for another launch), the exchanges are copies."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2605_02888_b200 as speckv
+from paper_2605_02888_b200 import synth, vocab_shard
+
+from parity import compare_step, gpu_batch, mlp_pair, oracle_batch
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _both(w, n_shards, step=0, bits=False):
+    s = synth.make_step(w, step, DEV)
+    gm, om = mlp_pair(synth.make_mlp(w, DEV))
+    out = vocab_shard.step_emulated(gpu_batch(s, entropy_in_bits=bits), n_shards, s["comp"], gm)
+    torch.cuda.synchronize()
+    ref = oracle.step(oracle_batch(s, entropy_in_bits=bits), s["comp"].cpu().numpy(), om)
+    return s, out, ref
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("n_shards", [1, 2, 3, 5])
+def test_small_vocabularies_ragged_last_shard(dtype, n_shards):
+    for V in (97, 1000, 4099):
+        w = synth.Workload("t", B=12, gamma_max=6, V=V, dtype=dtype, gamma_mode="ragged", temperature_mode="mixed",
+                           sigma_t=1.5, sigma_d=synth.SIGMA_LEVELS, frac_onehot=0.15, frac_identical=0.1, seed=V + n_shards)
+        for step in range(2):
+            s, out, ref = _both(w, n_shards, step)
+            compare_step(out, ref)
+
+
+@pytest.mark.parametrize("name,B,n_shards", [("b256", 24, 4), ("b512_mixed", 12, 8), ("b1024_loop", 16, 2)])
+def test_workloads_full_vocabulary(name, B, n_shards):
+    w = synth.scaled(synth.WORKLOADS[name], B=B)
+    s, out, ref = _both(w, n_shards)
+    rep = compare_step(out, ref)
+    assert rep["rows"] == B
+
+
+def test_matches_the_unsharded_step_and_entropy_in_bits():
+    w = synth.scaled(synth.WORKLOADS["b256"], B=16, V=32000)
+    s, out, ref = _both(w, 4, bits=True)
+    compare_step(out, ref)
+    gm, _ = mlp_pair(synth.make_mlp(w, DEV))
+    one = speckv.speckv_step(gpu_batch(s, entropy_in_bits=True), s["comp"], gm)
+    for k in ("n_accepted", "gamma_next", "row_status"):
+        assert torch.equal(out[k], one[k]), k
+    # signals: same statistics merged in another order
+    np.testing.assert_allclose(out["H"].cpu().numpy(), one["H"].cpu().numpy(), rtol=2e-6, atol=1e-7)
+    np.testing.assert_allclose(out["C"].cpu().numpy(), one["C"].cpu().numpy(), rtol=2e-6, atol=1e-7)
+
+
+def test_flagged_rows_and_token_in_every_shard():
+    w = synth.Workload("t", B=10, gamma_max=4, V=2048, dtype="fp32", gamma_mode="ragged", temperature=0.7,
+                       sigma_d=(1.0,), seed=11)
+    s = synth.make_step(w, 0, DEV)
+    s["gamma"][:] = 4                       # every planted position is a used one
+    s["draft_tokens"][0, 0] = 2047          # last shard
+    s["draft_tokens"][1, 0] = 0             # first shard
+    s["draft_tokens"][2, 1] = 5000          # outside the vocabulary -> flagged
+    s["gamma"][3] = 0                       # bad gamma
+    s["target"][4, 1, 700] = float("nan")   # non-finite, second shard of four
+    s["temperature"][5] = -1.0
+    gm, om = mlp_pair(synth.make_mlp(w, DEV))
+    out = vocab_shard.step_emulated(gpu_batch(s), 4, s["comp"], gm)
+    torch.cuda.synchronize()
+    ref = oracle.step(oracle_batch(s), s["comp"].cpu().numpy(), om)
+    compare_step(out, ref)
+    assert (ref["row_status"][[2, 3, 4, 5]] != 0).all() and (ref["row_status"][[0, 1]] == 0).all()
+
+
+def test_bounds_helper():
+    width, b = vocab_shard.shard_bounds(128256, 8)
+    assert width == 16032 and b[0] == (0, 16032) and b[-1] == (7 * 16032, 128256)
+    width, b = vocab_shard.shard_bounds(97, 3)
+    assert width == 40 and b[-1] == (80, 97)
+    with pytest.raises(ValueError):
+        vocab_shard.shard_bounds(16, 5)
