@@ -393,13 +393,17 @@ ShardPlan make_shard_plan(const speckv_batch* bt) {
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
     size_t off = 0;
-    p.off_tick = off; off = align_up(off + 2 * B * sizeof(int));  // sweep tickets, draw tickets
+    p.off_tick = off; off = align_up(off + (3 * B + 4) * sizeof(int));  // sweep tickets, draw tickets, counters, row queue
     p.off_part = off; off = align_up(off + B * J * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
     p.off_csum2 = off; off = align_up(off + B * p.nchunk * sizeof(float));
     p.total = off < kAlign ? kAlign : off;
     return p;
 }
+
+#ifndef SPECKV_SHARD_WARP_ROW_BYTES
+#define SPECKV_SHARD_WARP_ROW_BYTES 65536  // slice rows up to this size are swept by one warp each
+#endif
 
 // what every shard call needs from the local batch
 speckv_status shard_params(const speckv_batch* bt, void* ws, size_t ws_bytes, KParams& P, ShardPlan& pl) {
@@ -419,6 +423,10 @@ speckv_status shard_params(const speckv_batch* bt, void* ws, size_t ws_bytes, KP
     char* w = static_cast<char*>(ws);
     P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
     P.tick2 = P.tick1 + P.B;
+    P.qcount = P.tick1 + 2 * P.B;
+    P.qhead = P.qcount + 1;
+    P.qtail = P.qcount + 2;
+    P.rowq = P.qcount + 4;
     P.part = reinterpret_cast<float4*>(w + pl.off_part);
     P.csum = reinterpret_cast<float*>(w + pl.off_csum);
     P.csum2 = reinterpret_cast<float*>(w + pl.off_csum2);
@@ -549,12 +557,29 @@ speckv_status speckv_shard_sweep(const speckv_batch* local, int64_t v_begin, flo
     P.state = reinterpret_cast<float4*>(shard_state);
     P.tokl = reinterpret_cast<float2*>(shard_tokl);
     cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemsetAsync(P.tick1, 0, static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+    if (cudaMemsetAsync(P.tick1, 0, (3 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
+        return SPECKV_ERR_CUDA;
     if (cudaMemsetAsync(shard_tokl, 0, static_cast<size_t>(P.B) * P.G * sizeof(float2), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(P.n_sweep);
     constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
     const bool al = shard_aligned(local);
+    // A slice row is short (V / n_shards columns).  One CTA per short row is mostly overhead and the
+    // ring sweep pays per logit row as well (segment hand-over to its epilogue warp), so rows of up to
+    // 64 KB are swept by one warp each, all of them resident at once; wider slices take the
+    // CTA-per-slice sweep.
+    const long long row_bytes = static_cast<long long>(P.V) * esize(local->dtype);
+    if (row_bytes <= SPECKV_SHARD_WARP_ROW_BYTES) {
+        const unsigned g2 = static_cast<unsigned>((static_cast<long long>(P.B) * P.J + kWarps - 1) / kWarps);
+        if (local->dtype == SPECKV_BF16) {
+            if (al) shard_rows_kernel<__nv_bfloat16, true, Ub><<<g2, kThreads, 0, cs>>>(P);
+            else shard_rows_kernel<__nv_bfloat16, false, Ub><<<g2, kThreads, 0, cs>>>(P);
+        } else {
+            if (al) shard_rows_kernel<float, true, Uf><<<g2, kThreads, 0, cs>>>(P);
+            else shard_rows_kernel<float, false, Uf><<<g2, kThreads, 0, cs>>>(P);
+        }
+        return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+    }
     if (local->dtype == SPECKV_BF16) {
         if (al) sweep_kernel<__nv_bfloat16, true, Ub><<<grid, kThreads, 0, cs>>>(P);
         else sweep_kernel<__nv_bfloat16, false, Ub><<<grid, kThreads, 0, cs>>>(P);

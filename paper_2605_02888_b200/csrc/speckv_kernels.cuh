@@ -519,7 +519,9 @@ __device__ __forceinline__ Raw<T> ld_vec(const T* p) {
 // lane.  Lane l owns vectors l, l+32, ... of the range; U of them are in flight.  Warps of a
 // CTA never wait for one another.
 // ----------------------------------------------------------------------------------------
-template <typename T, bool ALIGNED, int PATH, int U, int STEP>
+// CTA_WARM: the warps of the CTA sweep slices of the same row and share their warm starts (one
+// barrier, every warp of the CTA must call); false: the warp is on its own row.
+template <typename T, bool ALIGNED, int PATH, int U, int STEP, bool CTA_WARM = true>
 __device__ __forceinline__ float4 sweep_warp(const T* __restrict__ row, int lo, int hi, int first, float scale,
                                              volatile float* sh_m0) {
     // this thread owns vectors first, first+STEP, ... of the range [lo, hi)
@@ -552,10 +554,12 @@ __device__ __forceinline__ float4 sweep_warp(const T* __restrict__ row, int lo, 
     }
     m0 = warp_maxf(m0);
     // share the warm start across the CTA's warps (one barrier per CTA, before the streaming loop)
-    if ((threadIdx.x & 31) == 0) sh_m0[threadIdx.x >> 5] = m0;
-    __syncthreads();
+    if (CTA_WARM) {
+        if ((threadIdx.x & 31) == 0) sh_m0[threadIdx.x >> 5] = m0;
+        __syncthreads();
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) m0 = fmaxf(m0, sh_m0[w]);
+        for (int w = 0; w < kWarps; ++w) m0 = fmaxf(m0, sh_m0[w]);
+    }
 
     DraftState ds; TargetState ts; ArgmaxState as;
     if constexpr (PATH == PATH_DRAFT) ds.init(m0);
@@ -961,11 +965,12 @@ __device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, f
     if (P.status && lane == 0) P.status[b] = status;
 }
 
-// Epilogue of a vocabulary shard's sweep (one warp per batch row): lane i merges this shard's partials
-// of draft position i and of target position i and writes the two merged states; the row epilogue
-// proper runs later on the states of all shards.  An argmax index becomes a global vocabulary index.
-__device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd,
-                                             const float4* pt, int n) {
+// Epilogue of a vocabulary shard's sweep (one warp per batch row): lane i merges this shard's nd
+// partials of draft position i and nt partials of target position i (the counts may differ from lane
+// to lane) and writes the two merged states; the row epilogue proper runs later on the states of all
+// shards.  An argmax index becomes a global vocabulary index.
+__device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd, int nd,
+                                             const float4* pt, int nt) {
     const int lane = threadIdx.x & 31;
     const int G = P.G;
     const bool ok = (gam >= 1 && gam <= G) && (Tf >= 0.f) && (Tf != __int_as_float(0x7f800000));
@@ -974,17 +979,17 @@ __device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, f
     float4* out = P.state + static_cast<long long>(b) * P.J;
     if (lane < G) {
         float4 ad = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ok && lane < gam) {
+        if (ok && lane < gam && nd > 0) {
             ad = ldcg4(pd);
-            for (int k = 1; k < n; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
+            for (int k = 1; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
         }
         out[G + 1 + lane] = ad;
     }
     if (lane <= G) {
         float4 at = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (ok && lane <= gam) {
+        if (ok && lane <= gam && nt > 0) {
             at = ldcg4(pt);
-            for (int k = 1; k < n; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
+            for (int k = 1; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k)) : merge_target(at, ldcg4(pt + k));
             if (greedy) {
                 const int idx = __float_as_int(at.y);
                 if (idx != 0x7fffffff) at.y = __int_as_float(idx + P.v_begin);
@@ -1113,7 +1118,8 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
         return;
     }
     if (P.export_state) {
-        export_epilogue(P, b, gam, Tf, P.part + (row0 + P.G + 1 + lane) * P.nsplit, P.part + (row0 + lane) * P.nsplit, P.nsplit);
+        export_epilogue(P, b, gam, Tf, P.part + (row0 + P.G + 1 + lane) * P.nsplit, P.nsplit,
+                           P.part + (row0 + lane) * P.nsplit, P.nsplit);
         return;
     }
     row_epilogue<T>(P, b, gam, Tf, P.part + (row0 + (verify ? P.G + 1 + lane : lane)) * P.nsplit, P.nsplit,

@@ -16,6 +16,50 @@
 
 namespace speckv {
 
+// Phase 1 for short slice rows: one warp per (batch row, logit row), every warp on its own row with
+// U loads of 16 bytes in flight per lane; the warp's merged state is the shard's state of that row.
+// No partials, no tickets.  (Wider slices use sweep_kernel with export_state set.)
+template <typename T, bool ALIGNED, int U>
+__global__ void __launch_bounds__(kThreads, SPECKV_MINB) shard_rows_kernel(const __grid_constant__ KParams P) {
+    const int lane = threadIdx.x & 31;
+    const long long w = static_cast<long long>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
+    if (w >= static_cast<long long>(P.B) * P.J) return;
+    const int b = static_cast<int>(w / P.J), j = static_cast<int>(w - static_cast<long long>(b) * P.J);
+    const int gam = P.gamma ? P.gamma[b] : P.G;
+    const float Tf = P.temp ? P.temp[b] : P.temp_scalar;
+    const bool row_ok = (gam >= 1 && gam <= P.G) && (Tf >= 0.f) && (Tf != __int_as_float(0x7f800000));
+    const bool greedy = (Tf == 0.f);
+    const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
+    const bool is_target = j <= P.G;
+    const int pos = is_target ? j : j - (P.G + 1);
+    const bool active = row_ok && (is_target ? pos <= gam : pos < gam);
+    float4 st = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (active) {
+        if (is_target) {
+            const T* row = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(pos) * P.tsp;
+            if (greedy) {
+                st = sweep_warp<T, ALIGNED, PATH_ARGMAX, U, 32, false>(row, 0, P.V, lane, scale, nullptr);
+                const int idx = __float_as_int(st.y);
+                if (idx != 0x7fffffff) st.y = __int_as_float(idx + P.v_begin);
+            } else {
+                st = sweep_warp<T, ALIGNED, PATH_TARGET, U, 32, false>(row, 0, P.V, lane, scale, nullptr);
+            }
+        } else {
+            const T* row = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb + static_cast<long long>(pos) * P.dsp;
+            if (lane == 0 && !greedy) {
+                // both logits at the draft token, if it falls into this slice
+                const int x = __ldg(P.tok + static_cast<long long>(b) * P.G + pos) - P.v_begin;
+                if (x >= 0 && x < P.V) {
+                    const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(pos) * P.tsp;
+                    P.tokl[static_cast<long long>(b) * P.G + pos] = make_float2(elem_to_float(row, x), elem_to_float(trow, x));
+                }
+            }
+            st = sweep_warp<T, ALIGNED, PATH_DRAFT, U, 32, false>(row, 0, P.V, lane, scale, nullptr);
+        }
+    }
+    if (lane == 0) P.state[static_cast<long long>(b) * P.J + j] = st;
+}
+
 // Phase 2: one warp per batch row; the partials of a logit row are the n_shards gathered states.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) shard_finish_kernel(const __grid_constant__ KParams P) {

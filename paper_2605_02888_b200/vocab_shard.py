@@ -134,3 +134,86 @@ def step_emulated(full: speckv.Batch, n_shards: int, comp: Optional[torch.Tensor
     toks = torch.stack([bf.out.out_tokens for bf in bufs]).max(dim=0).values
     bufs[0].out.out_tokens.copy_(toks)
     return bufs[0].out.as_dict()
+
+
+def main():
+    """Times one rank's four calls on its slice of a synthetic workload (one device; the exchanges
+    are copies of this rank's own buffers, so only their sizes are reported)."""
+    import argparse
+    import json
+
+    from . import synth
+
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="b256")
+    ap.add_argument("--shards", type=int, default=8)
+    ap.add_argument("--rank", type=int, default=0)
+    ap.add_argument("--rows", type=int, default=None)
+    ap.add_argument("--iters", type=int, default=50)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device: the library has no CPU path")
+    dev = torch.device("cuda", 0)
+    w = synth.WORKLOADS[args.workload]
+    if args.rows:
+        w = synth.scaled(w, B=args.rows)
+    s = synth.make_step(w, 0, dev)
+    width, bounds = shard_bounds(w.V, args.shards)
+    a, e = bounds[args.rank]
+    # a rank of a tensor-parallel projection holds its slice contiguously
+    local = speckv.Batch(draft_logits=s["draft"][:, :, a:e].contiguous(), target_logits=s["target"][:, :, a:e].contiguous(),
+                         draft_tokens=s["draft_tokens"], gamma=s["gamma"], temperature=s["temperature"],
+                         uniforms=s["uniforms"])
+    full = speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],
+                        gamma=s["gamma"], temperature=s["temperature"], uniforms=s["uniforms"])
+    mw = synth.make_mlp(w, dev)
+    mlp = speckv.Mlp(mw["W1"], mw["b1"], mw["W2"], mw["b2"])
+    # states of the other shards: computed once, from views of the full logits
+    others = []
+    for r, (ra, re) in enumerate(bounds):
+        b = ShardBuffers.allocate(slice_batch(full, ra, re), args.shards, mlp.n_out)
+        speckv.speckv_shard_sweep(slice_batch(full, ra, re), ra, b.state, b.tokl, b.workspace)
+        others.append(b)
+    buf = ShardBuffers.allocate(local, args.shards, mlp.n_out)
+    for r, o in enumerate(others):
+        buf.all_state[r].copy_(o.state)
+        buf.all_tokl[r].copy_(o.tokl)
+    speckv.speckv_shard_finish(local, args.shards, width, w.V, buf.all_state, buf.all_tokl, s["comp"], mlp, buf.out,
+                               buf.row_info)
+    for r, (o, (ra, re)) in enumerate(zip(others, bounds)):
+        speckv.speckv_shard_draw_sums(slice_batch(full, ra, re), buf.row_info, o.weight, o.workspace)
+        buf.all_weight[r].copy_(o.weight)
+    torch.cuda.synchronize()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.iters)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for it in range(args.iters + 3):
+        flush.zero_()                                   # the slice is smaller than L2: evict it between iterations
+        e5 = ev[max(it - 3, 0)]
+        e5[0].record()
+        speckv.speckv_shard_sweep(local, a, buf.state, buf.tokl, buf.workspace)
+        e5[1].record()
+        speckv.speckv_shard_finish(local, args.shards, width, w.V, buf.all_state, buf.all_tokl, s["comp"], mlp, buf.out,
+                                   buf.row_info)
+        e5[2].record()
+        speckv.speckv_shard_draw_sums(local, buf.row_info, buf.weight, buf.workspace)
+        e5[3].record()
+        speckv.speckv_shard_draw_pick(local, a, args.rank, args.shards, buf.row_info, buf.all_weight, buf.out.out_tokens,
+                                      buf.workspace)
+        e5[4].record()
+    torch.cuda.synchronize()
+    us = [1e3 * sum(e5[k].elapsed_time(e5[k + 1]) for e5 in ev) / args.iters for k in range(4)]
+    slice_bytes = int((2 * s["gamma"].long() + 1).sum()) * (e - a) * w.elem_bytes
+    B, G = w.B, w.gamma_max
+    print(json.dumps({
+        "workload": w.name, "rows": B, "shards": args.shards, "rank": args.rank, "slice_columns": e - a,
+        "us": {"sweep": us[0], "finish": us[1], "draw_sums": us[2], "draw_pick": us[3], "total": sum(us)},
+        "slice_logit_bytes": slice_bytes, "sweep_GBps": slice_bytes / us[0] / 1e3,
+        "exchanged_bytes_per_rank": {"states": B * (2 * G + 1) * 16, "token_logits": B * G * 8, "weights": B * 16,
+                                     "tokens": B * (G + 1) * 4},
+        "gathering_the_logits_instead_bytes_per_rank": slice_bytes,
+        "l2": "a 256 MB buffer is overwritten before every iteration"}))
+
+
+if __name__ == "__main__":
+    main()
