@@ -370,7 +370,8 @@ def speckv_step(batch: Batch, comp: Optional[torch.Tensor], mlp: Mlp, out: Optio
                 events: Optional[tuple] = None):
     """Fused step: signals + controller + verification.  Returns the StepOutputs tensors.
     `events`: optional (before_sweep, after_sweep, after_resample) torch.cuda.Event objects
-    (created with enable_timing=True); they are recorded around the two kernels."""
+    (created with enable_timing=True); they are recorded before and after the sweep kernel and after
+    the resample kernel (the last two coincide where the sweep kernel's grid draws the tokens itself)."""
     L = load_library()
     c = batch._c()
     m = mlp._c()

@@ -117,7 +117,7 @@ void fill_mlp(KParams& P, const speckv_mlp* m, const float* comp) {
     for (int j = 0; j < 8; ++j) P.gch[j] = m->gamma_choices[j];
 }
 
-struct Events {  // optional timing events around the two kernels
+struct Events {  // optional timing events around the kernels of a step
     cudaEvent_t before_sweep = nullptr, after_sweep = nullptr, after_resample = nullptr;
 };
 
@@ -261,9 +261,10 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     // the staged sweep wants whole 16-byte granules per row and a batch its per-row tables can hold
     const long long row_bytes = static_cast<long long>(P.V) * es;
     // Which sweep.  Measured on B200 (full-size workloads, same inputs): fp32 logits are bound by
-    // memory and the bulk-copy ring is faster (6.7-6.8 against 6.4 TB/s); bf16 logits need one
-    // exponential per two bytes and are bound by the special-function pipe, where the
-    // register-staged kernel with its 32 warps per SM hides latency better (4.95 against 4.6 TB/s).
+    // memory and the bulk-copy ring is faster (6.7-6.9 against 6.4 TB/s); bf16 logits need one
+    // exponential per two bytes, and hiding that latency next to the memory latency takes the 32
+    // warps per SM of the register-staged kernel (4.95 against 4.6 TB/s), whose draining tail the
+    // resample CTAs of the same grid then fill.
 #ifndef SPECKV_STAGED
 #define SPECKV_STAGED 1  // 0: never, 1: fp32 only, 2: whenever the layout allows (measurement builds)
 #endif

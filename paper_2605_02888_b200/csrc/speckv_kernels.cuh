@@ -5,11 +5,15 @@
 //   sweep kernel    one CTA per (row b, logit row j, vocabulary slice s).  Each thread keeps
 //                   an online-softmax state over 16-byte vector loads, the CTA merges the
 //                   256 states and stores one partial.  The last CTA of a batch row to finish
-//                   (found with a ticket counter, nobody waits) merges that row's partials in
-//                   double precision and writes signals, acceptance, controller outputs.
-//   resample kernel R CTAs per batch row rescan the stop position's draft/target rows, write
+//                   (found with a ticket counter, nobody waits) merges that row's partials,
+//                   decides the acceptances, raises the row's completion flag and then writes
+//                   the signals and the controller outputs.
+//   resample work   R CTAs per batch row rescan the stop position's draft/target rows, write
 //                   per-256-element chunk sums of the residual weights, and the last of them
-//                   locates the inverse-CDF threshold and writes the fresh token.
+//                   locates the inverse-CDF threshold and writes the fresh token.  These CTAs
+//                   sit behind the sweep CTAs in the sweep kernel's own grid and wait (bounded)
+//                   for their row's flag, or run as a kernel of their own after the ring sweep
+//                   of speckv_pipeline.cuh.
 #pragma once
 
 #include <cuda_bf16.h>
