@@ -390,6 +390,24 @@ def test_results_are_deterministic(name):
                                b[k].view(torch.int32) if b[k].dtype == torch.float32 else b[k]), k
 
 
+def test_full_size_step_repeats_bit_for_bit_with_one_workspace():
+    # the fresh tokens are drawn by CTAs that wait for a row's completion flag while other rows are still
+    # being swept: a missed ordering would show as a run that differs, or as a row flagged TIMEOUT
+    w = synth.WORKLOADS["b256"]
+    s = synth.make_step(w, 0, DEV)
+    gm, _ = mlp_pair(synth.make_mlp(w, DEV))
+    bt = gpu_batch(s)
+    out = speckv.StepOutputs.allocate(bt, gm.n_out)
+    first = {k: v.clone() for k, v in speckv.speckv_step(bt, s["comp"], gm, out=out).items()}
+    assert int(first["row_status"].abs().sum()) == 0
+    assert int((first["out_tokens"][torch.arange(w.B), first["n_accepted"].long()] < 0).sum()) == 0
+    for _ in range(40):
+        again = speckv.speckv_step(bt, s["comp"], gm, out=out)
+        for k, v in first.items():
+            assert torch.equal(v.view(torch.int32) if v.dtype == torch.float32 else v,
+                               again[k].view(torch.int32) if again[k].dtype == torch.float32 else again[k]), k
+
+
 def test_empty_batch_and_argument_errors():
     d = torch.zeros(0, 4, 100, device=DEV)
     out = speckv.speckv_signals(speckv.Batch(draft_logits=d))
