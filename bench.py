@@ -355,7 +355,9 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "B_per_gpu": w.B, "gamma_max": w.gamma_max, "V": w.V,
                        "logits": w.dtype, "temperature": w.temperature,
-                       "gamma_per_row": "hash-uniform over {2,4,6,8}", "mean_gamma": float(gam.float().mean()),
+                       "gamma_per_row": {"choices": "hash-uniform over {2,4,6,8}", "ragged": "hash-uniform over 1..gamma_max"}.get(
+                           w.gamma_mode, f"{min(w.gamma_fixed, w.gamma_max)} for every row"),
+                       "temperature_mode": w.temperature_mode, "mean_gamma": float(gam.float().mean()),
                        "l2": f"{n_batches} resident batches of {bytes_step[0] / 1e6:.0f} MB alternate (each larger than L2)",
                        "parallelism": f"dp{world} (rows sharded, no collective)"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,

@@ -66,6 +66,9 @@ WORKLOADS = {
                     gamma_fixed=4, temperature=1.0, sigma_t=2.0, sigma_d=SIGMA_LEVELS),
     "b256": Workload("b256", B=256, gamma_max=8, V=128256, dtype="bf16", steps=1, gamma_mode="choices",
                      temperature=0.8, sigma_t=2.5, sigma_d=SIGMA_LEVELS, frac_identical=0.10),
+    # the same batch with every row at gamma = 8: the upper end of the headline configuration's traffic
+    "b256_g8": Workload("b256_g8", B=256, gamma_max=8, V=128256, dtype="bf16", steps=1, gamma_mode="fixed",
+                        gamma_fixed=8, temperature=0.8, sigma_t=2.5, sigma_d=SIGMA_LEVELS, frac_identical=0.10),
     "b512_mixed": Workload("b512_mixed", B=512, gamma_max=8, V=151936, dtype="fp32", steps=1,
                            gamma_mode="choices", temperature_mode="mixed", sigma_t=2.0, sigma_d=(0.5,),
                            frac_onehot=0.05),
