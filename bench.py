@@ -268,10 +268,10 @@ def main():
     bytes_avg = sum(bytes_step[i % n_batches] for i in range(n_prof)) / n_prof
     peak, peak_kind = measured_hbm_peak()
     achieved = bytes_avg / (sweep_avg * 1e-3) / 1e9
-    # the library picks by logit type: fp32 -> ring sweep, then a resample kernel (two launches per step);
+    # the library picks by logit type and batch: fp32, 384..1024 rows -> ring sweep, then a resample kernel (two launches per step);
     # bf16 -> register-staged sweep whose grid also carries the resample CTAs (one launch per step, so
     # its duration is that of the whole pass over the batch, second read of the stop positions included)
-    kernel = "pipe_sweep_kernel" if w.dtype == "fp32" else "sweep_kernel"
+    kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024) else "sweep_kernel"
     one_launch = kernel == "sweep_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,

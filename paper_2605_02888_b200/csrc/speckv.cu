@@ -268,8 +268,14 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
 #ifndef SPECKV_STAGED
 #define SPECKV_STAGED 1  // 0: never, 1: fp32 only, 2: whenever the layout allows (measurement builds)
 #endif
+    // Below a few hundred rows the ring's fixed costs (per-CTA tables, one epilogue warp per CTA, a
+    // resample kernel that cannot overlap) outweigh its streaming rate: b512_mixed cut to 128 / 256 /
+    // 512 rows takes 178 / 317 / 564 us with the ring and 166 / 307 / 581 us without.
+#ifndef SPECKV_PIPE_MINB
+#define SPECKV_PIPE_MINB 384
+#endif
     const bool staged = (SPECKV_STAGED == 2 || (SPECKV_STAGED == 1 && bt->dtype == SPECKV_F32)) && aligned &&
-                        row_bytes % 16 == 0 && P.B <= kPipeMaxB;
+                        row_bytes % 16 == 0 && P.B <= kPipeMaxB && (SPECKV_STAGED == 2 || P.B >= SPECKV_PIPE_MINB);
     // completion flags per batch row and the logits at the draft tokens: only the register-staged sweep
     // overlaps the resample work with its own tail; after the ring sweep the resample kernel starts when
     // everything is done and a flag would only cost it a round trip
