@@ -1165,13 +1165,43 @@ __device__ __forceinline__ float rs_weight(const RsConst& c, float xt, float xd)
     return fmaxf(__fsub_rn(p, q), 0.f);
 }
 
+// A lane's kVec elements of a 256-element chunk.  bf16: eight adjacent elements (one 16-byte load, the warp
+// reads 512 contiguous bytes).  fp32: four adjacent elements of the chunk's first half and four of its
+// second half, so that each of the two loads of the warp covers 512 contiguous bytes (with eight
+// adjacent floats per lane every 32-byte sector would be requested twice).  rs_elem gives the vocabulary
+// index of element j.
+template <typename T>
+__device__ __forceinline__ int rs_elem(int chunk, int lane, int j) {
+    if constexpr (sizeof(T) == 2) return chunk * kChunk + lane * kVec + j;
+    else return chunk * kChunk + (j < kVec / 2 ? lane * (kVec / 2) + j : kChunk / 2 + lane * (kVec / 2) + j - kVec / 2);
+}
+template <bool ALIGNED>
+__device__ __forceinline__ uint4 rs_load4(const float* row, int e, int hi, float pad) {
+    if (ALIGNED && e + 4 <= hi) return ldg_stream(row + e);
+    float x[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) x[j] = (e + j < hi) ? row[e + j] : pad;
+    return make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
+}
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ Raw<T> rs_load_lane(const T* row, int chunk, int V, float pad) {
+    const int lane = threadIdx.x & 31;
+    if constexpr (sizeof(T) == 2) {
+        return load_raw<T, ALIGNED>(row, chunk * kChunk + lane * kVec, V, pad);
+    } else {
+        Raw<T> r;
+        r.a = rs_load4<ALIGNED>(row, chunk * kChunk + lane * 4, V, pad);
+        r.b = rs_load4<ALIGNED>(row, chunk * kChunk + kChunk / 2 + lane * 4, V, pad);
+        return r;
+    }
+}
+
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ void rs_load(const RsConst& c, const T* trow, const T* drow, int chunk, int V,
                                         Raw<T>& rt, Raw<T>& rd) {
-    const int e0 = chunk * kChunk + (threadIdx.x & 31) * kVec;
     const float ninf = __int_as_float(0xff800000);
-    rt = load_raw<T, ALIGNED>(trow, e0, V, ninf);
-    if (c.mode == RS_RESIDUAL) rd = load_raw<T, ALIGNED>(drow, e0, V, ninf);
+    rt = rs_load_lane<T, ALIGNED>(trow, chunk, V, ninf);
+    if (c.mode == RS_RESIDUAL) rd = rs_load_lane<T, ALIGNED>(drow, chunk, V, ninf);
     else rd = raw_fill<T>(ninf);
 }
 
@@ -1225,10 +1255,9 @@ __device__ __forceinline__ void rs_load_batch(const T* trow, const T* drow, int 
 #pragma unroll
     for (int u = 0; u < KU; ++u) {
         const int ch = base + u * kWarps;
-        const int e0 = ch * kChunk + (threadIdx.x & 31) * kVec;
         if (ch < c1) {
-            rt[u] = load_raw<T, ALIGNED>(trow, e0, V, ninf);
-            if (MODE == RS_RESIDUAL) rd[u] = load_raw<T, ALIGNED>(drow, e0, V, ninf);
+            rt[u] = rs_load_lane<T, ALIGNED>(trow, ch, V, ninf);
+            if (MODE == RS_RESIDUAL) rd[u] = rs_load_lane<T, ALIGNED>(drow, ch, V, ninf);
         } else {
             rt[u] = raw_fill<T>(ninf);
             if (MODE == RS_RESIDUAL) rd[u] = rt[u];
@@ -1358,25 +1387,32 @@ __device__ __forceinline__ int rs_search(const RsConst& c, const T* trow, const 
     // recompute the chunk's weights (bit-identical to the first pass) and scan them
     float w[kVec];
     rs_chunk_weights<T, ALIGNED>(c, trow, drow, chunk, V, w);
-    double lane_tot = 0.0;
-#pragma unroll
-    for (int j = 0; j < kVec; ++j) lane_tot += static_cast<double>(w[j]);
-    double lincl = lane_tot;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        double v = __shfl_up_sync(0xffffffffu, lincl, o);
-        if (lane >= o) lincl += v;
-    }
-    double run = before + (lincl - lane_tot);
+    // a lane's elements form one run of the chunk (bf16) or two (fp32, see rs_elem): scan run by run
+    constexpr int kSeg = sizeof(T) == 2 ? 1 : 2, kSegLen = kVec / kSeg;
     int found = 0x7fffffff, lastw = -1;
+    double seg_base = before;
 #pragma unroll
-    for (int j = 0; j < kVec; ++j) {
-        run += static_cast<double>(w[j]);
-        const int idx = chunk * kChunk + lane * kVec + j;
-        if (w[j] > 0.f) {
-            lastw = idx;
-            if (run > tau && found == 0x7fffffff) found = idx;
+    for (int sg = 0; sg < kSeg; ++sg) {
+        double lane_tot = 0.0;
+#pragma unroll
+        for (int j = 0; j < kSegLen; ++j) lane_tot += static_cast<double>(w[sg * kSegLen + j]);
+        double lincl = lane_tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            double v = __shfl_up_sync(0xffffffffu, lincl, o);
+            if (lane >= o) lincl += v;
         }
+        double run = seg_base + (lincl - lane_tot);
+#pragma unroll
+        for (int j = 0; j < kSegLen; ++j) {
+            run += static_cast<double>(w[sg * kSegLen + j]);
+            const int idx = rs_elem<T>(chunk, lane, sg * kSegLen + j);
+            if (w[sg * kSegLen + j] > 0.f) {
+                lastw = max(lastw, idx);
+                if (run > tau && found == 0x7fffffff) found = idx;
+            }
+        }
+        seg_base += __shfl_sync(0xffffffffu, lincl, 31);  // the whole run
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
