@@ -409,6 +409,34 @@ def test_full_size_step_repeats_bit_for_bit_with_one_workspace():
                                again[k].view(torch.int32) if again[k].dtype == torch.float32 else again[k]), k
 
 
+@pytest.mark.parametrize("name,B,V", [("b256", 64, 32000), ("b512_mixed", 400, 8000), ("b512_mixed", 32, 8000)])
+def test_step_can_be_captured_in_a_cuda_graph(name, B, V):
+    # the library only enqueues work on the caller's stream (no allocation, no synchronisation), so a step
+    # can be recorded once and replayed: single-launch path, ring sweep + dependent resample kernel, fp32 fallback
+    w = synth.scaled(synth.WORKLOADS[name], B=B, V=V)
+    s = synth.make_step(w, 0, DEV)
+    gm, _ = mlp_pair(synth.make_mlp(w, DEV))
+    bt = gpu_batch(s)
+    out = speckv.StepOutputs.allocate(bt, gm.n_out)
+    direct = {k: v.clone() for k, v in speckv.speckv_step(bt, s["comp"], gm, out=out).items()}
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        speckv.speckv_step(bt, s["comp"], gm, out=out)          # warm-up on the capturing stream
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            speckv.speckv_step(bt, s["comp"], gm, out=out)
+    for _ in range(3):
+        for v in out.as_dict().values():
+            v.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for k, v in direct.items():
+            assert torch.equal(v.view(torch.int32) if v.dtype == torch.float32 else v,
+                               out.as_dict()[k].view(torch.int32) if v.dtype == torch.float32 else out.as_dict()[k]), k
+
+
 def test_empty_batch_and_argument_errors():
     d = torch.zeros(0, 4, 100, device=DEV)
     out = speckv.speckv_signals(speckv.Batch(draft_logits=d))
