@@ -154,6 +154,9 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
 #ifndef SPECKV_RS_TAIL_MULT
 #define SPECKV_RS_TAIL_MULT 2
 #endif
+#ifndef SPECKV_RS_SMALL_CTAS
+#define SPECKV_RS_SMALL_CTAS 1184  // resample CTAs wanted in flight for a small batch (two per CTA slot)
+#endif
 #ifndef SPECKV_MERGED
 #define SPECKV_MERGED 1
 #endif
@@ -228,6 +231,17 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     P.nvec = pl.nvec;
     P.per_split = (pl.nvec + P.nsplit - 1) / P.nsplit;
     P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
+    {
+        // small batches: more, shorter shares per row, so that the draw of a handful of rows still spreads
+        // over the SMs (the draw of a row is a chain of dependent round trips, shorter with fewer chunks per CTA)
+        const int want = (SPECKV_RS_SMALL_CTAS + P.B - 1) / P.B;
+        int cap = (P.nchunk + 7) / 8;  // at least one chunk per warp
+        if (cap > 32) cap = 32;
+        if (want > P.R && cap > P.R) {
+            P.R = want < cap ? want : cap;
+            P.chunks_per_cta = (P.nchunk + P.R - 1) / P.R;
+        }
+    }
     P.mode = mode; P.bits = bt->entropy_in_bits ? 1 : 0;
     P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
     P.t = bt->target_logits; P.tsb = bt->target_stride_b; P.tsp = bt->target_stride_pos;
