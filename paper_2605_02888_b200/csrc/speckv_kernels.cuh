@@ -732,22 +732,24 @@ __device__ __forceinline__ double log2_split(double z) {
 // End of a row epilogue (whole warp): everything the warp wrote for batch row b becomes visible
 // before the row's completion flag does.  The resample kernel polls the flag instead of waiting for
 // the whole sweep grid, so it can work on finished rows while the sweep's last CTAs drain.
-__device__ __forceinline__ void row_done_signal(const KParams& P, int b) {
+__device__ __forceinline__ void row_done_signal(const KParams& P, int b, int mode, int n) {
     if (!P.rdone) return;
     __threadfence();
     __syncwarp();
-    if ((threadIdx.x & 31) == 0) asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(P.rdone + b), "r"(1) : "memory");
+    // the flag carries what a resample CTA needs to start fetching logits: draw mode and stop position
+    const int v = 1 | (mode << 8) | (n << 16);
+    if ((threadIdx.x & 31) == 0) asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(P.rdone + b), "r"(v) : "memory");
 }
 
-// Bounded wait for a row's completion flag (one thread polls).  False when the bound ran out.
-__device__ __forceinline__ bool row_done_wait(const int* flag) {
+// Bounded wait for a row's completion flag (one thread polls).  The flag's value, 0 when the bound ran out.
+__device__ __forceinline__ int row_done_wait(const int* flag) {
     for (int it = 0; it < (1 << 20); ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-        if (v) return true;
+        if (v) return v;
         __nanosleep(it < 64 ? 100 : 1000);
     }
-    return false;
+    return 0;
 }
 
 // Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
@@ -868,6 +870,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     const unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);  // first rejected position
     const int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
 
+    const int rs_mode = (verify && status == 0 && !greedy) ? (n < gam ? RS_RESIDUAL : RS_BONUS) : RS_NONE;
     if (verify) {
         // fresh token: known here for greedy rows, drawn by the resample step otherwise
         const int amax_n = __shfl_sync(0xffffffffu, amax, n);
@@ -885,7 +888,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         if (lane == 0) {
             P.n_acc[b] = n;
             RowInfo ri;
-            ri.mode = (status == 0 && !greedy) ? (n < gam ? RS_RESIDUAL : RS_BONUS) : RS_NONE;
+            ri.mode = rs_mode;
             ri.n = n;
             ri.u2 = (status == 0 && !greedy) ? u2_n : 0.f;
             ri.scale = scale;
@@ -895,7 +898,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         }
     }
     if (P.status && lane == 0) P.status[b] = status;
-    row_done_signal(P, b);
+    row_done_signal(P, b, rs_mode, n);
 
     // signals
     const float in_bits = P.bits ? static_cast<float>(kLog2e) : 1.f;
@@ -1265,15 +1268,18 @@ __device__ __forceinline__ void rs_load_batch(const T* trow, const T* drow, int 
     }
 }
 
-template <typename T, bool ALIGNED, int MODE, int KU>
-__device__ __forceinline__ void rs_chunk_sums_mode(RsConst c, const T* trow, const T* drow, int c0, int c1,
+// make_const() yields the row's constants; it is called after the first batch of loads has been issued,
+// so constants that are themselves still on their way from memory do not hold the loads up.
+template <typename T, bool ALIGNED, int MODE, int KU, class F>
+__device__ __forceinline__ void rs_chunk_sums_mode(F make_const, const T* trow, const T* drow, int c0, int c1,
                                                    int V, float* csum) {
-    c.mode = MODE;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int base = c0 + warp;
     if (base >= c1) return;
     Raw<T> rt[KU], rd[KU];
     rs_load_batch<T, ALIGNED, MODE, KU>(trow, drow, base, c1, V, rt, rd);
+    RsConst c = make_const();
+    c.mode = MODE;
     while (base < c1) {
         const int next = base + kWarps * KU;
         Raw<T> nt[KU], nd[KU];
@@ -1313,8 +1319,28 @@ __device__ __forceinline__ void rs_chunk_sums(const RsConst& c, const T* trow, c
                                               int V, float* csum) {
     constexpr int kResidual = sizeof(T) == 2 ? 2 : 1;  // chunks per batch: two rows to buffer
     constexpr int kBonus = 2;  // one row to buffer; measured: deeper bf16 batches leave a warp too few iterations
-    if (c.mode == RS_BONUS) rs_chunk_sums_mode<T, ALIGNED, RS_BONUS, kBonus>(c, trow, drow, c0, c1, V, csum);
-    else rs_chunk_sums_mode<T, ALIGNED, RS_RESIDUAL, kResidual>(c, trow, drow, c0, c1, V, csum);
+    auto mk = [&]() { return c; };
+    if (c.mode == RS_BONUS) rs_chunk_sums_mode<T, ALIGNED, RS_BONUS, kBonus>(mk, trow, drow, c0, c1, V, csum);
+    else rs_chunk_sums_mode<T, ALIGNED, RS_RESIDUAL, kResidual>(mk, trow, drow, c0, c1, V, csum);
+}
+
+// RowInfo as the two 16-byte words it is loaded as
+__device__ __forceinline__ RowInfo row_info_from(const int4& lo4, const int4& hi4) {
+    RowInfo ri;
+    ri.mode = lo4.x; ri.n = lo4.y; ri.u2 = __int_as_float(lo4.z); ri.scale = __int_as_float(lo4.w);
+    ri.lse2_p = __hiloint2double(hi4.y, hi4.x);
+    ri.lse2_q = __hiloint2double(hi4.w, hi4.z);
+    return ri;
+}
+// The same sums for a row whose mode is known but whose RowInfo words may still be in flight
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void rs_chunk_sums_info(int mode, const int4& lo4, const int4& hi4, const T* trow, const T* drow,
+                                                   int c0, int c1, int V, float* csum) {
+    constexpr int kResidual = sizeof(T) == 2 ? 2 : 1;
+    constexpr int kBonus = 2;
+    auto mk = [&]() { return rs_const(row_info_from(lo4, hi4), mode); };
+    if (mode == RS_BONUS) rs_chunk_sums_mode<T, ALIGNED, RS_BONUS, kBonus>(mk, trow, drow, c0, c1, V, csum);
+    else rs_chunk_sums_mode<T, ALIGNED, RS_RESIDUAL, kResidual>(mk, trow, drow, c0, c1, V, csum);
 }
 
 // The last CTA of a row copies the row's chunk sums into shared memory (one memory round trip for
@@ -1447,38 +1473,41 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     // summed while the sweep drains; every sweep CTA is resident or done before the first CTA of
     // this kernel starts, so the wait ends, and it is bounded all the same.  Without flags the CTA
     // waits for the whole sweep grid.
+    const int4* ip = reinterpret_cast<const int4*>(P.info + r);
+    int mode, n;
+    int4 lo4, hi4;
     if (P.rdone) {
-        if (threadIdx.x == 0) sh_flag = row_done_wait(P.rdone + b) ? 1 : 0;
+        if (threadIdx.x == 0) sh_flag = row_done_wait(P.rdone + b);
         __syncthreads();
-        if (!sh_flag) {
+        const int v = sh_flag;
+        if (!v) {
             if (threadIdx.x == 0 && share == 0 && P.status) atomicOr(P.status + b, 16);
             return;
         }
         __syncthreads();  // sh_flag is reused below
+        // mode and stop position came with the flag: the logit loads below can go out at once, the
+        // rest of the row's record (normalisers, second uniform) travels beside them
+        mode = (v >> 8) & 3;
+        n = v >> 16;
+        lo4 = __ldcg(ip); hi4 = __ldcg(ip + 1);
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
+        lo4 = __ldcg(ip); hi4 = __ldcg(ip + 1);
+        mode = lo4.x;
+        n = lo4.y;
     }
-    RowInfo ri;
-    {
-        const int4* ip = reinterpret_cast<const int4*>(P.info + r);
-        const int4 lo4 = __ldcg(ip), hi4 = __ldcg(ip + 1);
-        ri.mode = lo4.x; ri.n = lo4.y; ri.u2 = __int_as_float(lo4.z); ri.scale = __int_as_float(lo4.w);
-        ri.lse2_p = __hiloint2double(hi4.y, hi4.x);
-        ri.lse2_q = __hiloint2double(hi4.w, hi4.z);
-    }
-    if (ri.mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
-    const long long out_at = P.sample ? static_cast<long long>(r) : static_cast<long long>(b) * (P.G + 1) + ri.n;
+    if (mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
+    const long long out_at = P.sample ? static_cast<long long>(r) : static_cast<long long>(b) * (P.G + 1) + n;
 
     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
-                    static_cast<long long>(ri.n) * P.tsp;
+                    static_cast<long long>(n) * P.tsp;
     const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb +
-                    static_cast<long long>(ri.n) * P.dsp;
+                    static_cast<long long>(n) * P.dsp;
     float* csum = P.csum + static_cast<long long>(r) * P.nchunk;
-    RsConst c = rs_const(ri, ri.mode);
 
     const int c0 = share * cpc;
     const int c1 = min(P.nchunk, c0 + cpc);
-    rs_chunk_sums<T, ALIGNED>(c, trow, drow, c0, c1, P.V, csum);
+    rs_chunk_sums_info<T, ALIGNED>(mode, lo4, hi4, trow, drow, c0, c1, P.V, csum);
 
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -1491,6 +1520,8 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     __threadfence();
 
     // ---- last CTA of the row: locate the threshold ----
+    const RowInfo ri = row_info_from(__ldcg(ip), __ldcg(ip + 1));  // fetched again rather than kept in registers
+    RsConst c = rs_const(ri, mode);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int per_lane = (P.nchunk + 31) / 32;
     double own = 0.0, W = 0.0;
