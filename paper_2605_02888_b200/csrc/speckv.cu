@@ -320,7 +320,7 @@ SamplePlan make_sample_plan(const speckv_batch* bt) {
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
     size_t off = 0;
-    p.off_tick = off; off = align_up(off + (B + B * G) * sizeof(int));  // sweep tickets, resample tickets
+    p.off_tick = off; off = align_up(off + (2 * B + B * G) * sizeof(int));  // sweep tickets, resample tickets, row flags
     p.off_info = off; off = align_up(off + B * G * sizeof(RowInfo));
     p.off_part = off; off = align_up(off + B * G * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * G * p.nchunk * sizeof(float));
@@ -356,6 +356,7 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     char* w = static_cast<char*>(ws);
     P.tick1 = reinterpret_cast<int*>(w + pl.off_tick);
     P.tick2 = P.tick1 + P.B;
+    P.rdone = P.tick2 + static_cast<size_t>(P.B) * P.G;
     P.info = reinterpret_cast<RowInfo*>(w + pl.off_info);
     P.part = reinterpret_cast<float4*>(w + pl.off_part);
     P.csum = reinterpret_cast<float*>(w + pl.off_csum);
@@ -363,19 +364,24 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    const size_t n_tick = static_cast<size_t>(P.B) * (1 + static_cast<size_t>(P.G));
+    const size_t n_tick = static_cast<size_t>(P.B) * (2 + static_cast<size_t>(P.G));
     if (cudaMemsetAsync(P.tick1, 0, n_tick * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
     const int es = esize(bt->dtype);
     const bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
-    const unsigned grid1 = static_cast<unsigned>(P.B) * P.J * P.nsplit;
-    const unsigned grid2 = static_cast<unsigned>(P.B) * P.G * P.R;
+    // one launch: the draws' CTAs sit behind the sweep CTAs of the same grid and wait for their batch
+    // row's flag (as in the verification step); two launches when the grid would not fit
+    const long long n_draw = static_cast<long long>(P.B) * P.G * P.R;
+    const bool merged = SPECKV_MERGED && P.n_sweep + n_draw <= 0x7fffffffLL;
+    if (merged) P.rs_reverse = 0; else P.rdone = nullptr;
+    const unsigned grid1 = static_cast<unsigned>(P.n_sweep + (merged ? n_draw : 0));
+    const unsigned grid2 = static_cast<unsigned>(n_draw);
     constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
     if (bt->dtype == SPECKV_BF16) {
-        if (aligned) { sweep_kernel<__nv_bfloat16, true, Ub><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<__nv_bfloat16, true><<<grid2, kThreads, 0, cs>>>(P); }
-        else { sweep_kernel<__nv_bfloat16, false, Ub><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<__nv_bfloat16, false><<<grid2, kThreads, 0, cs>>>(P); }
+        if (aligned) { sweep_kernel<__nv_bfloat16, true, Ub><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<__nv_bfloat16, true><<<grid2, kThreads, 0, cs>>>(P); }
+        else { sweep_kernel<__nv_bfloat16, false, Ub><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<__nv_bfloat16, false><<<grid2, kThreads, 0, cs>>>(P); }
     } else {
-        if (aligned) { sweep_kernel<float, true, Uf><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<float, true><<<grid2, kThreads, 0, cs>>>(P); }
-        else { sweep_kernel<float, false, Uf><<<grid1, kThreads, 0, cs>>>(P); resample_kernel<float, false><<<grid2, kThreads, 0, cs>>>(P); }
+        if (aligned) { sweep_kernel<float, true, Uf><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<float, true><<<grid2, kThreads, 0, cs>>>(P); }
+        else { sweep_kernel<float, false, Uf><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<float, false><<<grid2, kThreads, 0, cs>>>(P); }
     }
     return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }

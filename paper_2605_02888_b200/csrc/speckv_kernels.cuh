@@ -970,6 +970,7 @@ __device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, f
         P.out_tok[r] = (ok && greedy) ? amax : -1;
     }
     if (P.status && lane == 0) P.status[b] = status;
+    row_done_signal(P, b, RS_NONE, 0);  // every position of the row has its own record: the flag only says they are written
 }
 
 // Epilogue of a vocabulary shard's sweep (one warp per batch row): lane i merges this shard's nd
@@ -1487,9 +1488,14 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
         __syncthreads();  // sh_flag is reused below
         // mode and stop position came with the flag: the logit loads below can go out at once, the
         // rest of the row's record (normalisers, second uniform) travels beside them
-        mode = (v >> 8) & 3;
-        n = v >> 16;
         lo4 = __ldcg(ip); hi4 = __ldcg(ip + 1);
+        if (P.sample) {  // one record per drafted position behind one flag per batch row
+            mode = lo4.x;
+            n = lo4.y;
+        } else {
+            mode = (v >> 8) & 3;
+            n = v >> 16;
+        }
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");
         lo4 = __ldcg(ip); hi4 = __ldcg(ip + 1);
