@@ -10,6 +10,7 @@
 #include "speckv_kernels.cuh"
 #include "speckv_pipeline.cuh"
 #include "speckv_shard.cuh"
+#include "speckv_sample.cuh"
 
 namespace {
 
@@ -309,7 +310,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
 // Draft-side sampling: its own workspace plan (one resample slot per drafted position).
 struct SamplePlan {
     int nchunk, R, chunks_per_cta;
-    size_t off_tick, off_info, off_part, off_csum, total;
+    size_t off_tick, off_info, off_part, off_csum, off_cz, total;
 };
 SamplePlan make_sample_plan(const speckv_batch* bt) {
     SamplePlan p;
@@ -324,6 +325,7 @@ SamplePlan make_sample_plan(const speckv_batch* bt) {
     p.off_info = off; off = align_up(off + B * G * sizeof(RowInfo));
     p.off_part = off; off = align_up(off + B * G * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * G * p.nchunk * sizeof(float));
+    p.off_cz = off; off = align_up(off + B * G * p.nchunk * sizeof(float2));  // per-chunk (maximum, sum) of the one-pass kernel
     p.total = off < kAlign ? kAlign : off;
     return p;
 }
@@ -368,6 +370,36 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     if (cudaMemsetAsync(P.tick1, 0, n_tick * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
     const int es = esize(bt->dtype);
     const bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
+#ifndef SPECKV_SAMPLE_CTAS
+#define SPECKV_SAMPLE_CTAS 2368
+#endif
+#ifndef SPECKV_SAMPLE_ONEPASS
+#define SPECKV_SAMPLE_ONEPASS 1  // 0: always normaliser sweep + second pass (measurement builds)
+#endif
+    // One pass (speckv_sample.cuh) whenever a row's chunk records fit the searching CTA's shared memory.
+    if (SPECKV_SAMPLE_ONEPASS && P.nchunk <= kRsStage &&
+        static_cast<long long>(P.B) * P.G * P.R <= 0x7fffffffLL) {
+        P.csum2 = reinterpret_cast<float*>(w + pl.off_cz);
+        // shares per logit row: enough CTAs to fill the SMs a few times over, no more (a CTA costs a few
+        // microseconds before its first load returns)
+        {
+            const long long draws = static_cast<long long>(P.B) * P.G;
+            long long S = (SPECKV_SAMPLE_CTAS + draws - 1) / draws;
+            if (S > P.R) S = P.R;
+            if (S < 1) S = 1;
+            P.R = static_cast<int>(S);
+            P.chunks_per_cta = (P.nchunk + P.R - 1) / P.R;
+        }
+        const unsigned g1 = static_cast<unsigned>(P.B) * P.G * P.R;
+        if (bt->dtype == SPECKV_BF16) {
+            if (aligned) sample_onepass_kernel<__nv_bfloat16, true><<<g1, kThreads, 0, cs>>>(P);
+            else sample_onepass_kernel<__nv_bfloat16, false><<<g1, kThreads, 0, cs>>>(P);
+        } else {
+            if (aligned) sample_onepass_kernel<float, true><<<g1, kThreads, 0, cs>>>(P);
+            else sample_onepass_kernel<float, false><<<g1, kThreads, 0, cs>>>(P);
+        }
+        return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+    }
     // one launch: the draws' CTAs sit behind the sweep CTAs of the same grid and wait for their batch
     // row's flag (as in the verification step); two launches when the grid would not fit
     const long long n_draw = static_cast<long long>(P.B) * P.G * P.R;
