@@ -241,6 +241,19 @@ def test_sample_draft_against_oracle(dtype, V):
     assert (s["temperature"] == 0).any() and (s["temperature"] > 0).any()
 
 
+def test_sample_draft_very_long_rows_take_the_two_pass_form():
+    # more chunks per row than the one-pass kernel stages: normaliser sweep, then the weights
+    w = synth.Workload("t", B=3, gamma_max=2, V=600_000, dtype="fp32", gamma_mode="fixed", gamma_fixed=2,
+                       temperature_mode="mixed", sigma_d=(0.5,), seed=33)
+    s = synth.make_step(w, 0, DEV)
+    u = torch.rand(w.B, w.gamma_max, device=DEV)
+    out = speckv.speckv_sample_draft(gpu_batch(s), u)
+    ref = oracle.sample_draft(oracle_batch(s), u.cpu().numpy())
+    np.testing.assert_array_equal(out["row_status"].cpu().numpy(), ref["row_status"])
+    bad = (out["tokens"].cpu().numpy() != ref["tokens"]).any(1)
+    assert not (bad & ((ref["near"] & oracle.NEAR_CDF) == 0)).any()
+
+
 def test_sample_draft_distribution_and_flags():
     rng = np.random.default_rng(8)
     V, N, T = 8, 200_000, 0.9
