@@ -12,6 +12,10 @@ import paper_2605_02888_b200 as speckv
 # bound for fp32 accumulation; ATOL covers entropies near zero, where 1e-5 relative of a value
 # like 1e-9 is below what fp32 sums of 10^5 terms can resolve.
 RTOL, ATOL = 1e-5, 1e-7
+# Controller scores (Eq. 1: E = a_hat * gamma + 1): a sum of terms of order one evaluated in fp32 as the task
+# statement fixes; where they cancel (E near 0) what is left is the rounding of the terms, a few units of
+# 2^-23 times gamma <= 8, so the absolute term is 1e-6 there.
+ATOL_SCORES = 1e-6
 
 
 def np_logits(t: torch.Tensor) -> np.ndarray:
@@ -92,7 +96,7 @@ def compare_step(gpu: dict, ref: dict, rows=None, check_controller=True, check_s
         assert np.all(g["out_tokens"][ok][cols.repeat(ok.sum(), 0) > g["n_accepted"][ok][:, None]] == -1)
         assert np.all(g["out_tokens"][ok][cols.repeat(ok.sum(), 0) <= g["n_accepted"][ok][:, None]] >= 0)
     if check_controller:
-        close(g["scores"], ref["scores"], "scores")
+        close(g["scores"], ref["scores"], "scores", atol=ATOL_SCORES)
         gm_bad = g["gamma_next"] != ref["gamma_next"]
         rep["near_gamma_rows"] = int(((near & oracle.NEAR_GAMMA) != 0).sum())
         rep["gamma_mismatch"] = int(gm_bad.sum())
