@@ -399,9 +399,17 @@ void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t*
         if (n < g) {
             std::vector<double> q(V);
             softmax_row(draft_row(bt, b, n), V, T, q.data());
-            for (int32_t v = 0; v < V; ++v) w[v] = std::max(0.0, p[v] - q[v]);
+            double Wres = 0.0;
+            for (int32_t v = 0; v < V; ++v) {
+                w[v] = std::max(0.0, p[v] - q[v]);
+                Wres += w[v];
+            }
             fresh = inverse_cdf(w.data(), V, u2, &nb);
             if (fresh < 0) fresh = inverse_cdf(p.data(), V, u2, &nb); /* p == q numerically */
+            /* A residual of total mass below 1e-5 (the probability that this rejection happens at all
+             * under the rule of Sec. 2.1) is beyond what weights held in fp32 resolve: such a draw is
+             * marked like a threshold on a boundary. */
+            if (Wres < 1e-5) nb = 1;
         } else {
             fresh = inverse_cdf(p.data(), V, u2, &nb);
         }

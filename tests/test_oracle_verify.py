@@ -282,3 +282,22 @@ def test_step_composes_signals_controller_and_verification():
     np.testing.assert_array_equal(s["scores"], ctl["scores"])
     np.testing.assert_array_equal(s["gamma_next"], ctl["gamma_next"])
     assert set(np.unique(s["gamma_next"])) <= {2, 4, 6, 8}
+
+
+def test_vanishing_residual_is_drawn_exactly_and_flagged():
+    # p and q agree to 1e-13 except on two far-tail tokens: the rejection of token 1 leaves a residual of
+    # total mass about 6e-14, all of it on token 2.  The rule still fixes the draw (token 2, whatever u' is);
+    # the row is marked, because weights held in fp32 cannot resolve such a residual.
+    d = np.array([[[0.0, -30.0, -31.0]]], np.float32)
+    t = np.array([[[0.0, -31.0, -30.0], [0.0, 0.0, 0.0]]], np.float32)
+    for u2 in (0.0, 0.3, 0.999):
+        u = np.array([[[0.9, u2], [0.5, 0.5]]], np.float32)
+        r = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=np.array([[1]], np.int32), uniforms=u))
+        assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 2
+        assert r["near"][0] & oracle.NEAR_CDF
+    # the same shape of problem with an ordinary residual is not marked
+    d2 = np.array([[[0.0, 1.0, -1.0]]], np.float32)
+    t2 = np.array([[[0.0, -1.0, 1.0], [0.0, 0.0, 0.0]]], np.float32)
+    r = oracle.verify(oracle.Batch(draft=d2, target=t2, draft_tokens=np.array([[1]], np.int32),
+                                   uniforms=np.array([[[0.9, 0.5], [0.5, 0.5]]], np.float32)))
+    assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 2 and not (r["near"][0] & oracle.NEAR_CDF)
