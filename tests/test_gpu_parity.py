@@ -450,6 +450,35 @@ def test_step_can_be_captured_in_a_cuda_graph(name, B, V):
                                out.as_dict()[k].view(torch.int32) if v.dtype == torch.float32 else out.as_dict()[k]), k
 
 
+def test_steps_overlapping_on_several_streams_match_their_serial_results():
+    # each call has its own workspace and outputs; the kernels of different calls share the SMs, among them
+    # CTAs that wait for a flag of their own grid and the persistent ring sweep
+    cfgs = [synth.scaled(synth.WORKLOADS["b256"], B=200), synth.scaled(synth.WORKLOADS["b512_mixed"], B=64, V=32000),
+            synth.scaled(synth.WORKLOADS["b1024_loop"], B=300, V=50000), synth.scaled(synth.WORKLOADS["b512_mixed"], B=400, V=16000)]
+    items = []
+    for w in cfgs:
+        s = synth.make_step(w, 0, DEV)
+        gm, _ = mlp_pair(synth.make_mlp(w, DEV))
+        bt = gpu_batch(s)
+        out = speckv.StepOutputs.allocate(bt, gm.n_out)
+        serial = {k: v.clone() for k, v in speckv.speckv_step(bt, s["comp"], gm, out=out).items()}
+        items.append((s, gm, bt, out, serial))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in items]
+    for _ in range(12):
+        for st, (s, gm, bt, out, serial) in zip(streams, items):
+            with torch.cuda.stream(st):
+                for v in out.as_dict().values():
+                    v.zero_()
+                speckv.speckv_step(bt, s["comp"], gm, out=out)
+        torch.cuda.synchronize()
+        for s, gm, bt, out, serial in items:
+            for k, v in serial.items():
+                a = out.as_dict()[k]
+                assert torch.equal(v.view(torch.int32) if v.dtype == torch.float32 else v,
+                                   a.view(torch.int32) if a.dtype == torch.float32 else a), k
+
+
 def test_empty_batch_and_argument_errors():
     d = torch.zeros(0, 4, 100, device=DEV)
     out = speckv.speckv_signals(speckv.Batch(draft_logits=d))
