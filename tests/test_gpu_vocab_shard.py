@@ -81,3 +81,38 @@ def test_bounds_helper():
     assert width == 40 and b[-1] == (80, 97)
     with pytest.raises(ValueError):
         vocab_shard.shard_bounds(16, 5)
+
+
+_ONE_RANK = r"""
+import os, sys, torch, torch.distributed as dist
+sys.path.insert(0, os.getcwd()); sys.path.insert(0, os.path.join(os.getcwd(), "tests"))
+os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=sys.argv[1], RANK="0", WORLD_SIZE="1")
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", rank=0, world_size=1)
+import paper_2605_02888_b200 as speckv
+from paper_2605_02888_b200 import synth, vocab_shard
+from parity import gpu_batch, mlp_pair
+w = synth.scaled(synth.WORKLOADS["b256"], B=12, V=16000)
+s = synth.make_step(w, 0, "cuda:0")
+gm, _ = mlp_pair(synth.make_mlp(w, "cuda:0"))
+bt = gpu_batch(s)
+width, bounds = vocab_shard.shard_bounds(w.V, 1)
+out = vocab_shard.step(bt, 0, width, w.V, s["comp"], gm)
+one = speckv.speckv_step(bt, s["comp"], gm)
+torch.cuda.synchronize()
+ok = all(torch.equal(out[k], one[k]) for k in ("n_accepted", "out_tokens", "gamma_next", "row_status"))
+dist.destroy_process_group()
+print("ONE_RANK_OK" if ok else "ONE_RANK_MISMATCH")
+"""
+
+
+def test_distributed_entry_runs_with_one_nccl_rank():
+    # the function a tensor-parallel job calls (all-gathers and the MAX all-reduce through NCCL), with the only
+    # process group a single GPU allows; several shards are covered above with the exchanges emulated
+    import os, socket, subprocess, sys
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", _ONE_RANK, str(port)], cwd=root, capture_output=True, text=True, timeout=300)
+    assert "ONE_RANK_OK" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
