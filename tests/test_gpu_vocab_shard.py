@@ -116,3 +116,22 @@ def test_distributed_entry_runs_with_one_nccl_rank():
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", _ONE_RANK, str(port)], cwd=root, capture_output=True, text=True, timeout=300)
     assert "ONE_RANK_OK" in r.stdout, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_argument_errors_are_reported_by_status():
+    w = synth.Workload("t", B=4, gamma_max=2, V=512, dtype="fp32", gamma_mode="fixed", gamma_fixed=2, sigma_d=(0.5,), seed=1)
+    s = synth.make_step(w, 0, DEV)
+    bt = gpu_batch(s)
+    buf = vocab_shard.ShardBuffers.allocate(bt, 2)
+    with pytest.raises(speckv.SpeckvError) as e:      # shard width that leaves the last shard empty
+        speckv.speckv_shard_finish(bt, 2, 512, 512, buf.all_state, buf.all_tokl, None, None, buf.out, buf.row_info)
+    assert e.value.code == 1
+    with pytest.raises(speckv.SpeckvError) as e:      # more shards than a warp has lanes
+        speckv.speckv_shard_draw_pick(bt, 0, 0, 33, buf.row_info, buf.all_weight, buf.out.out_tokens, buf.workspace)
+    assert e.value.code == 1
+    with pytest.raises(speckv.SpeckvError) as e:      # workspace too small
+        speckv.speckv_shard_sweep(bt, 0, buf.state, buf.tokl, buf.workspace[:256])
+    assert e.value.code == 3
+    with pytest.raises(speckv.SpeckvError) as e:      # rank outside the group
+        speckv.speckv_shard_draw_pick(bt, 0, 2, 2, buf.row_info, buf.all_weight, buf.out.out_tokens, buf.workspace)
+    assert e.value.code == 1
