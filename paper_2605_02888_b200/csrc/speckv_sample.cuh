@@ -3,8 +3,9 @@
 //
 // The inverse CDF needs the running sum of exp((x_v - M) / T) in vocabulary order, and M, the row
 // maximum, is known only at the end of the row.  Instead of a second pass, every 256-element chunk
-// keeps its own pair (m_c, Z_c = sum over the chunk of exp((x_v - m_c) / T)): rescaled by
-// exp((m_c - M) / T) these are the chunk sums the search needs, 8 bytes per 256 logits.  The CTA that
+// keeps a pair (m_c, Z_c = sum over the chunk of exp((x_v - m_c) / T)) with a reference m_c at or above
+// its elements: rescaled by exp((m_c - M) / T) these are the chunk sums the search needs, 8 bytes per
+// 256 logits.  The CTA that
 // completes a row stages the rescaled sums in shared memory, finds the chunk that holds u * Z and
 // reads that one chunk again.
 #pragma once
@@ -49,6 +50,7 @@ __global__ void __launch_bounds__(kThreads, 4) sample_onepass_kernel(const __gri
     const int c1 = min(P.nchunk, c0 + P.chunks_per_cta);
     constexpr int KU = sizeof(T) == 2 ? 4 : 2;  // chunks per batch: 16 registers of loads in flight per lane
     int base = c0 + warp;
+    float ref_m = ninf;  // sampled rows: the largest element this warp has met (the same in every lane)
     Raw<T> cur[KU];
 #pragma unroll
     for (int u = 0; u < KU; ++u)
@@ -73,8 +75,18 @@ __global__ void __launch_bounds__(kThreads, 4) sample_onepass_kernel(const __gri
                 if (x[j] < kFloor) x[j] = ninf;  // below the floor counts as -inf
                 lm = fmaxf(lm, x[j]);
             }
-            const float mc = warp_maxf(lm);
             bad = __any_sync(0xffffffffu, bad);
+            // The reference of a chunk's sum need not be the chunk's own maximum: any common value at or
+            // above it will do.  Sampled rows keep the warp's running maximum and raise it only when a lane
+            // sees a larger element (one vote per chunk instead of a five-step reduction); greedy rows need
+            // the chunk's maximum itself.
+            float mc;
+            if (greedy) {
+                mc = warp_maxf(lm);
+            } else {
+                if (__any_sync(0xffffffffu, lm > ref_m)) ref_m = fmaxf(ref_m, warp_maxf(lm));
+                mc = ref_m;
+            }
             float second;
             if (greedy) {
                 int idx = 0x7fffffff;
