@@ -26,7 +26,8 @@
  *   - inverse CDF in vocabulary order: smallest v with cumulative weight > u * total,
  *     falling back to the last v with positive weight;
  *   - argmax ties go to the lowest index (token id, and candidate gamma);
- *   - -inf logits are legal (probability 0); NaN, +inf or an all -inf row flag the row.
+ *   - -inf logits are legal (probability 0); NaN, +inf or an all -inf row flag the row;
+ *   - target rows behind the stop position are not part of the step: not read, not checked.
  */
 #include "speckv_oracle.h"
 
@@ -341,48 +342,62 @@ void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t*
     }
     const int32_t g = rp.gamma;
     const int32_t* xb = bt->draft_tokens + static_cast<int64_t>(b) * G;
+    /* What flags a row, in this order (a flagged row emits nothing):
+     *   a draft token outside [0, V)                       -> BAD_TOKEN;
+     *   a non-finite draft row at any drafted position     -> NONFINITE, and nothing else is looked at;
+     *   otherwise the positions are walked in order and the walk ends at the first position whose
+     *   target row is non-finite (-> NONFINITE), whose draft token is out of range, or whose token
+     *   is rejected.  Target rows behind that position are not part of the step: Sec. 3.1 emits the
+     *   accepted prefix and one token at the first mismatch and discards whatever the target
+     *   produced behind it, so those rows are neither read nor checked. */
     int32_t st = ORACLE_ROW_OK;
     for (int32_t i = 0; i < g; ++i)
         if (xb[i] < 0 || xb[i] >= V) st |= ORACLE_ROW_BAD_TOKEN;
+    const double Tq = (rp.T == 0.0) ? 1.0 : rp.T;
+    std::vector<double> mq(g), lzq(g);
+    bool draft_bad = false;
+    for (int32_t i = 0; i < g; ++i)
+        if (!lse_row(draft_row(bt, b, i), V, Tq, &mq[i], &lzq[i])) draft_bad = true;
+    if (draft_bad) {
+        if (row_status) row_status[b] |= st | ORACLE_ROW_NONFINITE;
+        return;
+    }
 
     int32_t n = g, fresh = -1, nearbits = 0;
 
     if (rp.T == 0.0) {
-        /* greedy rule of Sec. 3.1.  Every target row the step uses is checked first. */
-        std::vector<int32_t> am(g + 1);
+        /* greedy rule of Sec. 3.1 */
         for (int32_t i = 0; i <= g; ++i) {
-            am[i] = argmax_row(target_row(bt, b, i), V);
-            if (am[i] < 0) st |= ORACLE_ROW_NONFINITE;
-        }
-        for (int32_t i = 0; i < g; ++i)
-            if (argmax_row(draft_row(bt, b, i), V) < 0) st |= ORACLE_ROW_NONFINITE;
-        if (st) {
-            if (row_status) row_status[b] |= st;
-            return;
-        }
-        for (int32_t i = 0; i < g; ++i) {
-            if (xb[i] != am[i]) {
+            const int32_t am = argmax_row(target_row(bt, b, i), V);
+            if (am < 0) {
+                st |= ORACLE_ROW_NONFINITE;
+                break;
+            }
+            if (i < g && (xb[i] < 0 || xb[i] >= V)) break;
+            if (i == g || xb[i] != am) {
                 n = i;
+                fresh = am;
                 break;
             }
         }
-        fresh = am[n];
-    } else {
-        const double T = rp.T;
-        std::vector<double> mq(g), lzq(g), mp(g + 1), lzp(g + 1);
-        for (int32_t i = 0; i < g; ++i)
-            if (!lse_row(draft_row(bt, b, i), V, T, &mq[i], &lzq[i])) st |= ORACLE_ROW_NONFINITE;
-        for (int32_t i = 0; i <= g; ++i)
-            if (!lse_row(target_row(bt, b, i), V, T, &mp[i], &lzp[i])) st |= ORACLE_ROW_NONFINITE;
         if (st) {
             if (row_status) row_status[b] |= st;
             return;
         }
+    } else {
+        const double T = rp.T;
         const float* ub = bt->uniforms + static_cast<int64_t>(b) * (G + 1) * 2;
-        for (int32_t i = 0; i < g; ++i) {
+        for (int32_t i = 0; i <= g; ++i) {
+            double mp, lzp;
+            if (!lse_row(target_row(bt, b, i), V, T, &mp, &lzp)) {
+                st |= ORACLE_ROW_NONFINITE;
+                break;
+            }
+            if (i == g) break; /* every drafted token accepted */
+            if (xb[i] < 0 || xb[i] >= V) break;
             const double u = static_cast<double>(ub[2 * i + 0]);
             const double lnq = draft_row(bt, b, i).at(xb[i]) / T - mq[i] - lzq[i];
-            const double lnp = target_row(bt, b, i).at(xb[i]) / T - mp[i] - lzp[i];
+            const double lnp = target_row(bt, b, i).at(xb[i]) / T - mp - lzp;
             const double ratio = std::exp(lnp - lnq); /* p(x)/q(x); inf when q(x) = 0 < p(x) */
             if (std::fabs(u - ratio) < 1e-6) nearbits |= ORACLE_NEAR_ACCEPT;
             /* accept iff u*q(x) < p(x) */
@@ -391,6 +406,10 @@ void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t*
                 n = i;
                 break;
             }
+        }
+        if (st) {
+            if (row_status) row_status[b] |= st;
+            return;
         }
         std::vector<double> p(V), w(V);
         softmax_row(target_row(bt, b, n), V, T, p.data());
@@ -407,9 +426,9 @@ void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t*
             fresh = inverse_cdf(w.data(), V, u2, &nb);
             if (fresh < 0) fresh = inverse_cdf(p.data(), V, u2, &nb); /* p == q numerically */
             /* A residual of total mass below 1e-5 (the probability that this rejection happens at all
-             * under the rule of Sec. 2.1) is beyond what weights held in fp32 resolve: such a draw is
-             * marked like a threshold on a boundary. */
-            if (Wres < 1e-5) nb = 1;
+             * under the rule of Sec. 2.1) is beyond what weights held in fp32 resolve: the draw is
+             * exact here and the row carries a flag of its own. */
+            if (Wres < 1e-5) nearbits |= ORACLE_NEAR_SMALL_RESIDUAL;
         } else {
             fresh = inverse_cdf(p.data(), V, u2, &nb);
         }

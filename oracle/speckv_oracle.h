@@ -37,10 +37,10 @@ extern "C" {
 
 /* per-row near-tie bits (rows where a comparison is closer than the stated margin) */
 #define ORACLE_NEAR_ACCEPT 1 /* |u - p(x)/q(x)| < 1e-6 at a tested position            */
-#define ORACLE_NEAR_CDF 2    /* inverse-CDF threshold within 1e-6*W of a boundary, or a  */
-                             /* residual of total mass below 1e-5                        */
+#define ORACLE_NEAR_CDF 2    /* inverse-CDF threshold within 1e-6*W of a boundary        */
 #define ORACLE_NEAR_GREEDY 4 /* (unused for exact ties: those resolve by lowest index)   */
 #define ORACLE_NEAR_GAMMA 8  /* best and second-best controller score within 1e-5 rel.   */
+#define ORACLE_NEAR_SMALL_RESIDUAL 16 /* rejected position whose residual mass is below 1e-5 */
 
 typedef struct {
     int32_t B;         /* rows (sequences) in the batch                                  */

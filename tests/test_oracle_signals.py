@@ -187,3 +187,41 @@ def test_status_flags():
     r = oracle.signals(oracle.Batch(draft=x, temperature=np.array([-1, 1, 1, 1, np.nan], np.float32)))
     assert r["row_status"][0] == oracle.ROW_BAD_TEMPERATURE
     assert r["row_status"][4] == oracle.ROW_BAD_TEMPERATURE
+
+
+def _merge(a, b):
+    """Merge rule for two partial softmax states (m, Z, S) of disjoint parts of one row, with
+    Z = sum e^(x-m) and S = sum e^(x-m) (x-m): bring both to the common maximum and add."""
+    m = max(a[0], b[0])
+    out_z, out_s = 0.0, 0.0
+    for (mk, zk, sk) in (a, b):
+        f = math.exp(mk - m)
+        out_z += zk * f
+        out_s += f * (sk + (mk - m) * zk)
+    return (m, out_z, out_s)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_merging_random_partitions_reproduces_the_unsplit_signals(seed):
+    # H = ln Z - S/Z and c = 1/Z from states merged over a random partition of the row must equal the
+    # oracle's -sum q ln q and max q on the whole row (Sec. 4.2): this is the identity a split sweep rests on.
+    rng = np.random.default_rng(seed)
+    V, T = 5000 + 37 * seed, (1.0, 0.7, 1.3, 2.0)[seed]
+    x = rng.normal(0, 3, V).astype(np.float32)
+    x[rng.integers(0, V, 40)] = -np.inf            # masked tokens contribute nothing
+    ref = _sig(x[None, None, :], temperature_scalar=T)
+    cuts = np.sort(rng.choice(np.arange(1, V), size=int(rng.integers(1, 12)), replace=False))
+    parts = np.split(x.astype(np.float64) / float(np.float32(T)), cuts)
+    rng.shuffle(parts)                             # the merge is order-free
+    state = None
+    for part in parts:
+        fin = part[np.isfinite(part)]
+        if fin.size == 0:
+            continue
+        m = fin.max()
+        e = np.exp(fin - m)
+        st = (m, e.sum(), (e * (fin - m)).sum())
+        state = st if state is None else _merge(state, st)
+    m, Z, S = state
+    assert math.log(Z) - S / Z == pytest.approx(ref["H"][0, 0], rel=1e-12, abs=1e-12)
+    assert 1.0 / Z == pytest.approx(ref["C"][0, 0], rel=1e-12)

@@ -239,7 +239,7 @@ def test_row_status_flags_and_outputs():
     tok = rng.integers(0, V, (B, G)).astype(np.int32)
     tok[1, 2] = V
     tok[2, 0] = -1
-    t[3, 3, 4] = np.nan
+    t[3, 0, 4] = np.nan                     # position 0 is read whatever happens later
     gam = np.array([3, 3, 3, 3, 4, 2], np.int32)
     T = np.array([1, 1, 0, 1, 1, -0.5], np.float32)
     u = rng.random((B, G + 1, 2)).astype(np.float32)
@@ -294,10 +294,121 @@ def test_vanishing_residual_is_drawn_exactly_and_flagged():
         u = np.array([[[0.9, u2], [0.5, 0.5]]], np.float32)
         r = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=np.array([[1]], np.int32), uniforms=u))
         assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 2
-        assert r["near"][0] & oracle.NEAR_CDF
+        assert r["near"][0] & oracle.NEAR_SMALL_RESIDUAL
     # the same shape of problem with an ordinary residual is not marked
     d2 = np.array([[[0.0, 1.0, -1.0]]], np.float32)
     t2 = np.array([[[0.0, -1.0, 1.0], [0.0, 0.0, 0.0]]], np.float32)
     r = oracle.verify(oracle.Batch(draft=d2, target=t2, draft_tokens=np.array([[1]], np.int32),
                                    uniforms=np.array([[[0.9, 0.5], [0.5, 0.5]]], np.float32)))
-    assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 2 and not (r["near"][0] & oracle.NEAR_CDF)
+    assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 2 and not (r["near"][0] & (oracle.NEAR_CDF | oracle.NEAR_SMALL_RESIDUAL))
+
+
+def _four_token_case():
+    """gamma = 2, V = 4.  Draft = uniform; the three target rows put their excess mass on different
+    tokens, so that the residual of position i (and the bonus distribution of position 2) sits on a
+    token of its own: position 0 -> token 1, position 1 -> token 2, position 2 -> token 3."""
+    d = np.zeros((1, 2, 4), np.float32)
+    t = np.full((1, 3, 4), 0.0, np.float32)
+    t[0, 0, 1] = 3.0
+    t[0, 1, 2] = 3.0
+    t[0, 2, :] = [NEG, NEG, NEG, 0.0]          # bonus distribution: token 3 with probability 1
+    return d, t
+
+
+def test_second_uniform_is_taken_at_the_stop_position():
+    # Token 0 has p/q = 4 p(0) < 1 at both drafted positions (p(0) = 1 / (3 + e^3) = 0.043, ratio 0.173).
+    d, t = _four_token_case()
+    p1 = _softmax(t[0, 1])
+    assert 4 * p1[0] < 0.2
+    tok = np.zeros((1, 2), np.int32)
+    # residual of position 1 = max(0, p1 - 1/4): all of it on token 2; of position 0: all on token 1.
+    # Accept position 0 (u = 0.01 < 0.173), reject position 1 (u = 0.9).  The second uniforms differ per
+    # position; only u[b, 1, 1] may be consumed.  With a two-token residual the choice shows which one was.
+    t2 = t.copy()
+    t2[0, 1, :] = [0.0, 0.0, 2.0, 2.0]         # position 1: residual on tokens 2 and 3, equal halves
+    u = np.zeros((1, 3, 2), np.float32)
+    u[0, :, 0] = [0.01, 0.9, 0.5]
+    for u11, want in ((0.25, 2), (0.75, 3)):
+        for other in (0.25, 0.75):              # whatever the other positions' second uniforms say
+            u[0, :, 1] = [other, u11, other]
+            r = oracle.verify(oracle.Batch(draft=d, target=t2, draft_tokens=tok, uniforms=u))
+            assert r["n_accepted"][0] == 1
+            assert list(r["out_tokens"][0]) == [0, want, -1]
+    # rejected at position 0 instead: the residual there is token 1 only, and u[b, 0, 1] is the one read
+    u[0, :, 0] = [0.9, 0.01, 0.5]
+    u[0, :, 1] = [0.5, 0.25, 0.75]
+    r = oracle.verify(oracle.Batch(draft=d, target=t2, draft_tokens=tok, uniforms=u))
+    assert r["n_accepted"][0] == 0 and list(r["out_tokens"][0]) == [1, -1, -1]
+
+
+def test_bonus_draw_reads_the_second_uniform_of_position_gamma():
+    # both drafted tokens accepted (u = 0.01); the bonus row splits its mass over tokens 1 and 3
+    d, t = _four_token_case()
+    t[0, 2, :] = [NEG, 0.0, NEG, 0.0]
+    tok = np.zeros((1, 2), np.int32)
+    u = np.zeros((1, 3, 2), np.float32)
+    u[0, :, 0] = 0.01
+    for u21, want in ((0.25, 1), (0.75, 3)):
+        for other in (0.25, 0.75):
+            u[0, :, 1] = [other, other, u21]
+            r = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=tok, uniforms=u))
+            assert r["n_accepted"][0] == 2 and list(r["out_tokens"][0]) == [0, 0, want]
+
+
+def test_target_rows_behind_the_stop_position_are_not_part_of_the_step():
+    # Sec. 3.1: the step emits the accepted prefix and one token at the first mismatch.  A NaN in a target
+    # row behind the stop position changes nothing; at or before it, it flags the row.
+    d, t = _four_token_case()
+    tok = np.zeros((1, 2), np.int32)
+    u = np.zeros((1, 3, 2), np.float32)
+    u[0, :, 0] = [0.9, 0.01, 0.5]               # rejected at position 0
+    u[0, :, 1] = 0.5
+    clean = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=tok, uniforms=u))
+    assert clean["n_accepted"][0] == 0 and clean["row_status"][0] == 0
+    for pos, flagged in ((0, True), (1, False), (2, False)):
+        tt = t.copy()
+        tt[0, pos, 3] = np.nan
+        for T in (1.0, 0.0):                    # sampling rule and greedy rule (token 0 is never the argmax)
+            r = oracle.verify(oracle.Batch(draft=d, target=tt, draft_tokens=tok, uniforms=u, temperature_scalar=T))
+            assert (r["row_status"][0] == oracle.ROW_NONFINITE) == flagged, (pos, T)
+            if not flagged:
+                assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == 1
+    # a non-finite *draft* row flags the row wherever it is: the signals use every drafted position
+    dd = d.copy()
+    dd[0, 1, 2] = np.inf
+    r = oracle.verify(oracle.Batch(draft=dd, target=t, draft_tokens=tok, uniforms=u))
+    assert r["row_status"][0] == oracle.ROW_NONFINITE and r["out_tokens"][0, 0] == -1
+    # an out-of-range token ends the walk: a NaN behind it is not reached, one in front of it is
+    tok2 = np.array([[0, 7]], np.int32)
+    u[0, :, 0] = 0.01                           # position 0 accepted, position 1 cannot be tested
+    for pos, want in ((2, oracle.ROW_BAD_TOKEN), (1, oracle.ROW_BAD_TOKEN | oracle.ROW_NONFINITE),
+                      (0, oracle.ROW_BAD_TOKEN | oracle.ROW_NONFINITE)):
+        tt = t.copy()
+        tt[0, pos, 0] = np.nan
+        r = oracle.verify(oracle.Batch(draft=d, target=tt, draft_tokens=tok2, uniforms=u))
+        assert r["row_status"][0] == want, pos
+
+
+def test_step_gives_flagged_rows_neutral_outputs():
+    rng = np.random.default_rng(16)
+    B, G, V = 5, 3, 24
+    t = rng.normal(0, 1, (B, G + 1, V)).astype(np.float32)
+    d = rng.normal(0, 1, (B, G, V)).astype(np.float32)
+    tok = rng.integers(0, V, (B, G)).astype(np.int32)
+    gam = np.array([3, 0, 3, 3, 3], np.int32)    # row 1: bad gamma
+    tok[2, 1] = V + 3                            # row 2: bad token
+    d[3, 2, 5] = np.nan                          # row 3: NaN in a draft row
+    T = np.array([1, 1, 1, 1, np.nan], np.float32)  # row 4: bad temperature
+    u = rng.random((B, G + 1, 2)).astype(np.float32)
+    comp = np.zeros((B, 2), np.float32)
+    mlp = oracle.Mlp(rng.normal(0, 0.1, (16, 5)), rng.normal(0, 0.1, 16), rng.normal(0, 0.1, (4, 16)),
+                     rng.normal(0, 0.1, 4))
+    s = oracle.step(oracle.Batch(draft=d, target=t, draft_tokens=tok, gamma=gam, temperature=T, uniforms=u), comp, mlp)
+    assert list(s["row_status"]) == [0, oracle.ROW_BAD_GAMMA, oracle.ROW_BAD_TOKEN, oracle.ROW_NONFINITE,
+                                     oracle.ROW_BAD_TEMPERATURE]
+    for b in range(1, B):
+        assert s["n_accepted"][b] == 0 and np.all(s["out_tokens"][b] == -1)
+        assert s["gamma_next"][b] == 0 and np.all(s["scores"][b] == 0)
+        assert np.all(s["H"][b] == 0) and np.all(s["C"][b] == 0) and np.all(s["feat"][b] == 0)
+    # the healthy row is untouched by its neighbours
+    assert s["gamma_next"][0] in (2, 4, 6, 8) and s["feat"][0, 0] > 0 and s["out_tokens"][0, s["n_accepted"][0]] >= 0
