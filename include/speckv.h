@@ -31,7 +31,10 @@
  *     gamma_next = 0 and zeros in its float outputs.  No kernel traps; every wait inside a
  *     kernel is bounded and ends in SPECKV_ROW_TIMEOUT on the row at hand.
  *   - Logits below -2^100 are treated as -inf (probability 0).  NaN or +inf anywhere in a used
- *     logit row, or a used row without any finite entry, flags the row.
+ *     logit row, or a used row without any finite entry, flags the row.  Used rows are the draft
+ *     rows of all gamma_b drafted positions and the target rows up to the stop position (the first
+ *     position that is rejected, or gamma_b); target rows behind it are not part of the step
+ *     (Sec. 3.1) and flag nothing.
  *   - Temperature: 0 selects the greedy rule (and T = 1 for that row's signals); otherwise
  *     finite and >= 1e-6.
  */
@@ -85,7 +88,20 @@ typedef struct {
     const float* uniforms;   /* [B, gamma_max+1, 2] in [0,1): [b,i,0] accept test at i,   */
                              /* [b,n,1] resample at the stop position n (bonus: n=gamma_b) */
     int32_t entropy_in_bits; /* 0: nats; 1: bits (the paper's log2)                       */
+    int32_t flags;           /* SPECKV_* flags below, 0 for the defaults                  */
 } speckv_batch;
+
+/* speckv_batch.flags (verification calls; ignored by the others) */
+enum {
+    /* Read every target row 0..gamma_b of every batch row.  By default a target row behind a position
+     * that is already known to be rejected is left out: Sec. 3.1 discards what the target produced
+     * behind the first mismatch, so such a row changes no output.  Results are the same either way. */
+    SPECKV_READ_ALL_TARGET_ROWS = 1,
+    /* Scheduling hints (results are the same either way): take the stream kernel (persistent CTAs,
+     * position-major order) or the sliced sweep whatever the batch size.  At most one of the two.     */
+    SPECKV_SCHEDULE_STREAM = 2,
+    SPECKV_SCHEDULE_SLICED = 4
+};
 
 typedef struct {
     int32_t n_in, n_hidden, n_out; /* 5, 16, 4 in the primary form                        */
@@ -142,25 +158,14 @@ speckv_status speckv_sample_draft(const speckv_batch* batch, const float* unifor
                                   void* cuda_stream);
 
 /* One fused step: signals, controller and verification from a single pass over the logits
- * (plus a second look at the stop position's two rows for the residual / bonus draw).
+ * (plus a second look at the stop position's two rows for the residual / bonus draw, taken
+ * while those rows are still in L2 where the batch is large enough for the stream kernel).
  * gamma_next[b] is the controller's choice for the NEXT step of row b; this step verifies
  * with the gamma given in the batch.  H, C, scores may be NULL.                            */
 speckv_status speckv_step(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
                           float* H, float* C, float* feat, float* scores, int32_t* gamma_next,
                           int32_t* n_accepted, int32_t* out_tokens, int32_t* row_status,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
-
-/* Measurement aid: speckv_step with three caller-created CUDA events (cudaEvent_t passed as
- * void*) recorded on the stream before the sweep kernel, after it, and after the resample
- * kernel, so that a benchmark can time the dominant kernel alone.  Where the sweep kernel's own
- * grid draws the fresh tokens (bf16 logits) there is no resample kernel and the last two events
- * coincide.  Results are identical to speckv_step.  Any event may be NULL.                 */
-speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp, const speckv_mlp* mlp,
-                                   float* H, float* C, float* feat, float* scores,
-                                   int32_t* gamma_next, int32_t* n_accepted, int32_t* out_tokens,
-                                   int32_t* row_status, void* workspace, size_t workspace_bytes,
-                                   void* cuda_stream, void* ev_before_sweep, void* ev_after_sweep,
-                                   void* ev_after_resample);
 
 /* speckv_signals for callers that cannot allocate device memory.  (The paper has no counterpart:
  * this entry point exists for deployment reasons only.)

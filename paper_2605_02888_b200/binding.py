@@ -20,6 +20,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_STATIC_LIMIT 
 F32, BF16 = 0, 1
 ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE, ROW_TIMEOUT = 0, 1, 2, 4, 8, 16
 
+READ_ALL_TARGET_ROWS, SCHEDULE_STREAM, SCHEDULE_SLICED = 1, 2, 4   # speckv_batch.flags
+
 STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_signals_static", "speckv_select_gamma", "speckv_verify",
            "speckv_sample_workspace_size", "speckv_sample_draft",
@@ -37,7 +39,8 @@ class _CBatch(C.Structure):
                 ("draft_logits", C.c_void_p), ("draft_stride_b", C.c_int64), ("draft_stride_pos", C.c_int64),
                 ("target_logits", C.c_void_p), ("target_stride_b", C.c_int64), ("target_stride_pos", C.c_int64),
                 ("draft_tokens", C.c_void_p), ("gamma", C.c_void_p), ("temperature", C.c_void_p),
-                ("temperature_scalar", C.c_float), ("uniforms", C.c_void_p), ("entropy_in_bits", C.c_int32)]
+                ("temperature_scalar", C.c_float), ("uniforms", C.c_void_p), ("entropy_in_bits", C.c_int32),
+                ("flags", C.c_int32)]
 
 
 class _CMlp(C.Structure):
@@ -82,8 +85,13 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_verify.argtypes = [C.POINTER(_CBatch), vp, vp, vp, vp, sz, vp]
     L.speckv_step.restype = C.c_int
     L.speckv_step.argtypes = [C.POINTER(_CBatch), vp, C.POINTER(_CMlp)] + [vp] * 8 + [vp, sz, vp]
+    # include/speckv_internal.h: the benchmark's timing aid and two test hooks
     L.speckv_step_profiled.restype = C.c_int
     L.speckv_step_profiled.argtypes = L.speckv_step.argtypes + [vp, vp, vp]
+    L.speckv_internal_set_wait_limit.restype = C.c_int
+    L.speckv_internal_set_wait_limit.argtypes = [C.c_int]
+    L.speckv_internal_wait_probe.restype = C.c_int
+    L.speckv_internal_wait_probe.argtypes = [C.c_int32, vp, vp, vp, sz, vp]
     i32, i64 = C.c_int32, C.c_int64
     L.speckv_shard_workspace_size.restype = C.c_int
     L.speckv_shard_workspace_size.argtypes = [C.POINTER(_CBatch), C.POINTER(sz)]
@@ -135,6 +143,7 @@ class Batch:
     temperature_scalar: float = 1.0
     uniforms: Optional[torch.Tensor] = None         # [B, gamma_max+1, 2] fp32
     entropy_in_bits: bool = False
+    flags: int = 0                                  # READ_ALL_TARGET_ROWS | SCHEDULE_STREAM | SCHEDULE_SLICED
 
     def shape(self):
         B, G, V = self.draft_logits.shape
@@ -172,6 +181,7 @@ class Batch:
             setattr(c, name, _dev_ptr(a, dt, name))
         c.temperature_scalar = float(self.temperature_scalar)
         c.entropy_in_bits = int(bool(self.entropy_in_bits))
+        c.flags = int(self.flags)
         return c
 
 

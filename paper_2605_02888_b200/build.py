@@ -10,7 +10,8 @@ _CSRC = os.path.join(_PKG, "csrc")
 _INC = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_CSRC, "libspeckv.so")
 _SOURCES = ["speckv.cu"]
-_DEPS = ["speckv.cu", "speckv_kernels.cuh", "speckv_pipeline.cuh", "speckv_shard.cuh", "speckv_sample.cuh"]
+_DEPS = ["speckv.cu", "speckv_kernels.cuh", "speckv_pipeline.cuh", "speckv_shard.cuh", "speckv_sample.cuh",
+         "speckv_stream.cuh"]
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared"]
@@ -27,7 +28,7 @@ def is_stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(_CSRC, d) for d in _DEPS] + [os.path.join(_INC, "speckv.h")]
+    deps = [os.path.join(_CSRC, d) for d in _DEPS] + [os.path.join(_INC, h) for h in ("speckv.h", "speckv_internal.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

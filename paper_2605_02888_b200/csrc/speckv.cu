@@ -1,9 +1,14 @@
 // Host side of libspeckv: argument checks, workspace plan and kernel launches behind the
-// C ABI declared in include/speckv.h.  No allocation, no synchronisation, no global state.
+// C ABI declared in include/speckv.h.  No allocation, no synchronisation.  The only state the
+// library keeps between calls is a handful of per-device constants (SM count, kernel attributes set,
+// the address of the built-in scratch array), each published with release/acquire atomics; none of
+// them survives cudaDeviceReset.
 #include "speckv.h"
+#include "speckv_internal.h"
 
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 
@@ -11,6 +16,7 @@
 #include "speckv_pipeline.cuh"
 #include "speckv_shard.cuh"
 #include "speckv_sample.cuh"
+#include "speckv_stream.cuh"
 
 namespace {
 
@@ -20,6 +26,9 @@ using namespace speckv;
 #define SPECKV_SLICE_BYTES 262144 // bytes of one logit row that one sweep CTA streams
 #endif
 constexpr size_t kAlign = 256;
+// upper bound of a verification step's logit bytes from which the stream kernel is taken
+constexpr long long kStreamMinBytes = 128ll << 20;
+constexpr bool kStreamByDefault = false;  // until it outruns the sliced sweep on the large batches
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Plan {
@@ -75,6 +84,60 @@ Plan make_plan(const speckv_batch* bt) {
     return p;
 }
 
+// Workspace of the stream kernel (speckv_stream.cuh).  Depends on the batch shape only.
+struct StreamPlan {
+    bool fits;        // the shape is one the stream kernel takes
+    int n_slice, slice_elems, rs_shares, nchunk;
+    size_t off_ctrl, off_state, off_ptick, off_tick2, off_rsq, zero_bytes;  // [0, zero_bytes) is cleared per call
+    size_t off_info, off_pos, off_fresh, off_part, off_csum, total;
+};
+
+StreamPlan make_stream_plan(const speckv_batch* bt) {
+    StreamPlan p{};
+    const size_t B = static_cast<size_t>(bt->B), G1 = static_cast<size_t>(bt->gamma_max) + 1;
+    // slices per logit row: none for large batches; small batches are cut so that the SMs have a few
+    // items each; a slice holds at most kSMaxQ warp quanta
+    const long long max_slice = static_cast<long long>(kSMaxQ) * kSQElems;
+    long long ns = (bt->V + max_slice - 1) / max_slice;
+    const long long rows = static_cast<long long>(bt->B) * (2 * bt->gamma_max + 1);
+    const long long want = rows > 0 ? (4 * 148 + rows - 1) / rows : 1;
+    if (want > ns) ns = want;
+    if (ns > kSMaxSlice) ns = kSMaxSlice;
+    long long se = (bt->V + ns - 1) / ns;
+    se = (se + kSQElems - 1) / kSQElems * kSQElems;
+    ns = (bt->V + se - 1) / se;
+    p.n_slice = static_cast<int>(ns);
+    p.slice_elems = static_cast<int>(se);
+    p.nchunk = (bt->V + kChunk - 1) / kChunk;
+    p.rs_shares = (p.nchunk + kSRsShare - 1) / kSRsShare;
+    p.fits = bt->B <= kSMaxB && se <= max_slice && ns <= kSMaxSlice && bt->V <= (1 << 28) &&
+             static_cast<long long>(bt->B) * G1 * 2 * ns <= 0x7fffffffLL / 4;
+    size_t off = 0;
+    p.off_ctrl = off; off = align_up(off + sizeof(SCtrl));
+    p.off_state = off; off = align_up(off + B * sizeof(unsigned long long));
+    p.off_ptick = off; off = align_up(off + B * G1 * sizeof(int));
+    p.off_tick2 = off; off = align_up(off + B * sizeof(int));
+    p.off_rsq = off; off = align_up(off + B * sizeof(int));
+    p.zero_bytes = off;
+    p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
+    p.off_pos = off; off = align_up(off + B * G1 * sizeof(PosRec));
+    p.off_fresh = off; off = align_up(off + B * sizeof(int));
+    p.off_part = off; off = align_up(off + B * G1 * 2 * static_cast<size_t>(ns) * sizeof(float4));
+    p.off_csum = off; off = align_up(off + B * static_cast<size_t>(p.nchunk) * sizeof(float));
+    p.total = off;
+    return p;
+}
+
+// what the caller must provide: enough for whichever kernel the call takes
+size_t workspace_total(const speckv_batch* bt) {
+    const Plan a = make_plan(bt);
+    const StreamPlan b = make_stream_plan(bt);
+    return (b.fits && b.total > a.total) ? b.total : a.total;
+}
+
+// polls a waiting CTA spends before it gives a row up (SPECKV_ROW_TIMEOUT); lowered by tests only
+std::atomic<int> g_wait_limit{1 << 20};
+
 speckv_status check_batch(const speckv_batch* bt, bool need_target) {
     if (!bt) return SPECKV_ERR_INVALID_ARG;
     if (bt->B < 0 || bt->gamma_max < 1 || bt->V < 1) return SPECKV_ERR_INVALID_ARG;
@@ -91,6 +154,8 @@ speckv_status check_batch(const speckv_batch* bt, bool need_target) {
         if (!stride_ok(bt->target_stride_b) || !stride_ok(bt->target_stride_pos)) return SPECKV_ERR_INVALID_ARG;
     }
     if (!(bt->temperature) && !(bt->temperature_scalar >= 0.f)) return SPECKV_ERR_INVALID_ARG;
+    if (bt->flags & ~(SPECKV_READ_ALL_TARGET_ROWS | SPECKV_SCHEDULE_STREAM | SPECKV_SCHEDULE_SLICED)) return SPECKV_ERR_INVALID_ARG;
+    if ((bt->flags & SPECKV_SCHEDULE_STREAM) && (bt->flags & SPECKV_SCHEDULE_SLICED)) return SPECKV_ERR_INVALID_ARG;
     return SPECKV_OK;
 }
 
@@ -124,24 +189,40 @@ struct Events {  // optional timing events around the kernels of a step
 
 // Staged sweep: persistent CTAs, two per SM.  Needs 16-byte aligned rows whose byte length is a
 // multiple of 16, and a batch whose per-row tables fit in shared memory.
+// SM count of the current device, looked up once per device (0 in the slot = not yet known).
+cudaError_t sm_count(int* out) {
+    static std::atomic<int> cached[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool slot = dev >= 0 && dev < 64;
+    int sms = slot ? cached[dev].load(std::memory_order_acquire) : 0;
+    if (sms == 0) {
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        if (slot) cached[dev].store(sms, std::memory_order_release);
+    }
+    *out = sms;
+    return cudaSuccess;
+}
+
 template <typename T>
 cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
-    static bool configured[64] = {};
-    static int n_sm[64] = {};
+    static std::atomic<bool> configured[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     const size_t smem = (sizeof(PipeShared) + 127) / 128 * 128 + static_cast<size_t>(kStages) * kStageBytes;
     const bool slot = dev >= 0 && dev < 64;
-    int sms = slot ? n_sm[dev] : 0;
-    if (!slot || !configured[dev]) {
+    if (!slot || !configured[dev].load(std::memory_order_acquire)) {
         e = cudaFuncSetAttribute(pipe_sweep_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        if (slot) { n_sm[dev] = sms; configured[dev] = true; }
+        if (slot) configured[dev].store(true, std::memory_order_release);
     }
+    int sms = 0;
+    e = sm_count(&sms);
+    if (e != cudaSuccess) return e;
     pipe_sweep_kernel<T><<<SPECKV_PIPE_CTAS * sms, kPipeThreads, smem, st>>>(P);
     return cudaGetLastError();
 }
@@ -206,6 +287,20 @@ cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged
     return e;
 }
 
+// The stream kernel: one persistent CTA per SM (speckv_stream.cuh).
+template <typename T>
+cudaError_t launch_stream(const KParams& P, const SParams& S, cudaStream_t st, const Events& ev) {
+    int sms = 0;
+    cudaError_t e = sm_count(&sms);
+    if (e != cudaSuccess) return e;
+    if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
+    stream_kernel<T><<<sms, kSThreads, 0, st>>>(P, S);
+    e = cudaGetLastError();
+    if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
+    if (ev.after_resample) cudaEventRecord(ev.after_resample, st);
+    return e;
+}
+
 // Shared driver of signals / verify / step.
 speckv_status run(const speckv_batch* bt, int mode, const float* comp, const speckv_mlp* mlp, float* H,
                   float* C, float* feat, float* scores, int32_t* gamma_next, int32_t* n_accepted,
@@ -223,7 +318,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     if (bt->B == 0) return SPECKV_OK;
     const Plan pl = make_plan(bt);
     if (!ws || reinterpret_cast<uintptr_t>(ws) % kAlign != 0) return SPECKV_ERR_INVALID_ARG;
-    if (ws_bytes < pl.total) return SPECKV_ERR_WORKSPACE;
+    if (ws_bytes < workspace_total(bt)) return SPECKV_ERR_WORKSPACE;
 
     KParams P{};
     P.B = bt->B; P.G = bt->gamma_max; P.V = bt->V;
@@ -244,6 +339,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
         }
     }
     P.mode = mode; P.bits = bt->entropy_in_bits ? 1 : 0;
+    P.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
     P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
     P.t = bt->target_logits; P.tsb = bt->target_stride_b; P.tsp = bt->target_stride_pos;
     P.tok = bt->draft_tokens; P.gamma = bt->gamma; P.temp = bt->temperature;
@@ -266,15 +362,46 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    if (cudaMemsetAsync(P.tick1, 0, (4 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
-        return SPECKV_ERR_CUDA;
-
     const int es = esize(bt->dtype);
     bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
     if (verify) aligned = aligned && rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
+    const long long row_bytes = static_cast<long long>(P.V) * es;
+
+    // Verification of batches with enough logit rows to keep every SM streaming goes to the stream kernel
+    // (position-major order, early exit behind a rejection, draws from L2); smaller ones, signals alone
+    // and rows that are not whole 16-byte granules take the sliced sweep below.
+    {
+        const StreamPlan sp = make_stream_plan(bt);
+        const long long upper_bytes = static_cast<long long>(P.B) * pl.J_full * row_bytes;
+        const bool big = upper_bytes >= kStreamMinBytes;
+        const bool want = (bt->flags & SPECKV_SCHEDULE_STREAM) ||
+                          (kStreamByDefault && !(bt->flags & SPECKV_SCHEDULE_SLICED) && big && bt->dtype == SPECKV_BF16);
+        if (verify && want && sp.fits && aligned && row_bytes % 16 == 0) {
+            if (cudaMemsetAsync(ws, 0, sp.zero_bytes, cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+            SParams S{};
+            S.n_slice = sp.n_slice; S.slice_elems = sp.slice_elems; S.rs_shares = sp.rs_shares;
+            S.read_all = (bt->flags & SPECKV_READ_ALL_TARGET_ROWS) ? 1 : 0;
+            S.ctrl = reinterpret_cast<SCtrl*>(w + sp.off_ctrl);
+            S.state = reinterpret_cast<unsigned long long*>(w + sp.off_state);
+            S.ptick = reinterpret_cast<int*>(w + sp.off_ptick);
+            S.rsq = reinterpret_cast<int*>(w + sp.off_rsq);
+            S.pos = reinterpret_cast<PosRec*>(w + sp.off_pos);
+            S.fresh = reinterpret_cast<int*>(w + sp.off_fresh);
+            S.poll_limit = P.wait_limit;
+            P.tick2 = reinterpret_cast<int*>(w + sp.off_tick2);
+            P.info = reinterpret_cast<RowInfo*>(w + sp.off_info);
+            P.part = reinterpret_cast<float4*>(w + sp.off_part);
+            P.csum = reinterpret_cast<float*>(w + sp.off_csum);
+            const cudaError_t e = bt->dtype == SPECKV_BF16 ? launch_stream<__nv_bfloat16>(P, S, cs, ev)
+                                                          : launch_stream<float>(P, S, cs, ev);
+            return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
+        }
+    }
+
+    if (cudaMemsetAsync(P.tick1, 0, (4 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
+        return SPECKV_ERR_CUDA;
 
     // the staged sweep wants whole 16-byte granules per row and a batch its per-row tables can hold
-    const long long row_bytes = static_cast<long long>(P.V) * es;
     // Which sweep.  Measured on B200 (full-size workloads, same inputs): fp32 logits are bound by
     // memory and the bulk-copy ring is faster (6.7-6.9 against 6.4 TB/s); bf16 logits need one
     // exponential per two bytes, and hiding that latency next to the memory latency takes the 32
@@ -349,6 +476,7 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     P.per_split = (P.nvec + P.nsplit - 1) / P.nsplit;
     P.nchunk = pl.nchunk; P.R = pl.R; P.chunks_per_cta = pl.chunks_per_cta;
     P.mode = MODE_SAMPLE; P.sample = 1; P.rs_reverse = 1;
+    P.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
     // the drafted positions are swept and drawn from as if they were target rows
     P.d = bt->draft_logits; P.dsb = bt->draft_stride_b; P.dsp = bt->draft_stride_pos;
     P.t = bt->draft_logits; P.tsb = bt->draft_stride_b; P.tsp = bt->draft_stride_pos;
@@ -424,15 +552,17 @@ static __device__ __align__(256) unsigned char g_static_scratch[SPECKV_STATIC_SC
 // Device address of g_static_scratch on the current device.  In host code the array's name only
 // stands for the symbol; the address a kernel can use has to be asked for, once per device.
 cudaError_t static_scratch_address(void** out) {
-    static void* cached[64] = {};
+    static std::atomic<void*> cached[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64 && cached[dev]) { *out = cached[dev]; return cudaSuccess; }
-    void* p = nullptr;
-    e = cudaGetSymbolAddress(&p, g_static_scratch);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) cached[dev] = p;
+    const bool slot = dev >= 0 && dev < 64;
+    void* p = slot ? cached[dev].load(std::memory_order_acquire) : nullptr;
+    if (!p) {
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (slot) cached[dev].store(p, std::memory_order_release);
+    }
     *out = p;
     return cudaSuccess;
 }
@@ -497,6 +627,23 @@ bool shard_aligned(const speckv_batch* bt) {
            rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
 }
 
+// Kernels of speckv_internal_wait_probe: arbitrary status words and empty token slots before the draw
+// kernel runs, and afterwards a row epilogue that arrives late and raises each row's completion flag.
+__global__ void wait_probe_fill(KParams P) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= P.B) return;
+    P.status[b] = 0x5a5a;
+    P.out_tok[2 * b] = -1;
+    P.out_tok[2 * b + 1] = -1;
+}
+__global__ void wait_probe_late_epilogue(KParams P) {
+    const int b = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    if (b >= P.B) return;
+    if ((threadIdx.x & 31) == 0) P.status[b] = 0;
+    __syncwarp();
+    row_done_signal(P, b, RS_BONUS, 1);
+}
+
 }  // namespace
 
 extern "C" {
@@ -506,7 +653,7 @@ speckv_status speckv_workspace_size(const speckv_batch* batch, size_t* bytes) {
     if (!batch || batch->B < 0 || batch->gamma_max < 1 || batch->V < 1) return SPECKV_ERR_INVALID_ARG;
     if (batch->gamma_max > SPECKV_MAX_GAMMA || batch->V > (1 << 30) || batch->B > (1 << 24))
         return SPECKV_ERR_UNSUPPORTED;
-    *bytes = make_plan(batch).total;
+    *bytes = workspace_total(batch);
     return SPECKV_OK;
 }
 
@@ -589,6 +736,32 @@ speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp,
     ev.after_resample = static_cast<cudaEvent_t>(ev_after_resample);
     return run(batch, MODE_SIGNALS | MODE_VERIFY | MODE_MLP, comp, mlp, H, C, feat, scores, gamma_next,
                n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream, ev);
+}
+
+int speckv_internal_set_wait_limit(int polls) {
+    if (polls < 1) polls = 1;
+    return g_wait_limit.exchange(polls);
+}
+
+speckv_status speckv_internal_wait_probe(int32_t B, int32_t* row_status, int32_t* out_tokens, void* workspace,
+                                         size_t workspace_bytes, void* cuda_stream) {
+    if (B < 1 || B > 4096 || !row_status || !out_tokens || !workspace) return SPECKV_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(workspace) % kAlign != 0 || workspace_bytes < 2 * static_cast<size_t>(B) * sizeof(int))
+        return SPECKV_ERR_WORKSPACE;
+    // the draw kernel on its own, one CTA per batch row, with completion flags that nothing raises
+    KParams P{};
+    P.B = B; P.G = 1; P.V = kChunk; P.J = 3; P.nchunk = 1; P.R = 1; P.chunks_per_cta = 1;
+    P.R2 = 1; P.chunks_per_cta2 = 1; P.mode = MODE_VERIFY;
+    P.wait_limit = g_wait_limit.load(std::memory_order_relaxed);
+    P.status = row_status; P.out_tok = out_tokens;
+    P.rdone = static_cast<int*>(workspace);
+    P.tick2 = P.rdone + B;
+    cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(workspace, 0, 2 * static_cast<size_t>(B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
+    wait_probe_fill<<<(B + 255) / 256, 256, 0, cs>>>(P);
+    resample_kernel<float, true><<<static_cast<unsigned>(B), kThreads, 0, cs>>>(P);
+    wait_probe_late_epilogue<<<(B + kWarps - 1) / kWarps, kThreads, 0, cs>>>(P);
+    return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
 
 speckv_status speckv_shard_workspace_size(const speckv_batch* local, size_t* bytes) {

@@ -58,6 +58,7 @@ struct KParams {
     int n_sweep;  // sweep kernel: CTAs that sweep; the rest of the grid (if any) does the resample work
     int sample;  // 1: draft-side sampling (every drafted position draws a token from its own row)
     int rs_tail, R2, chunks_per_cta2;  // resample: the last rs_tail draws in launch order use R2 CTAs each
+    int wait_limit;  // polls a resample CTA spends on its row's completion flag before it gives the row up
     int rs_reverse;  // resample kernel: 1 = last batch row first (after a sweep it cannot overlap: those rows are the freshest in L2)
     int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
@@ -732,21 +733,27 @@ __device__ __forceinline__ double log2_split(double z) {
 // End of a row epilogue (whole warp): everything the warp wrote for batch row b becomes visible
 // before the row's completion flag does.  The resample kernel polls the flag instead of waiting for
 // the whole sweep grid, so it can work on finished rows while the sweep's last CTAs drain.
+constexpr int kRowDoneTimeout = 1 << 30;  // a resample CTA gave up waiting for this row
 __device__ __forceinline__ void row_done_signal(const KParams& P, int b, int mode, int n) {
     if (!P.rdone) return;
     __threadfence();
     __syncwarp();
     // the flag carries what a resample CTA needs to start fetching logits: draw mode and stop position
     const int v = 1 | (mode << 8) | (n << 16);
-    if ((threadIdx.x & 31) == 0) asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(P.rdone + b), "r"(v) : "memory");
+    if ((threadIdx.x & 31) == 0) {
+        const int old = atomicOr(P.rdone + b, v);
+        // a resample CTA whose bounded wait ran out before this point left its mark here: the row's fresh
+        // token will never be drawn, and the status written above must say so
+        if ((old & kRowDoneTimeout) && P.status) atomicOr(P.status + b, 16);
+    }
 }
 
 // Bounded wait for a row's completion flag (one thread polls).  The flag's value, 0 when the bound ran out.
-__device__ __forceinline__ int row_done_wait(const int* flag) {
-    for (int it = 0; it < (1 << 20); ++it) {
+__device__ __forceinline__ int row_done_wait(const int* flag, int limit) {
+    for (int it = 0; it < limit; ++it) {
         int v;
         asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-        if (v) return v;
+        if (v & 1) return v;
         __nanosleep(it < 64 ? 100 : 1000);
     }
     return 0;
@@ -813,7 +820,8 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
     float Hi = 0.f, ci = 0.f;
     double lse2_q = 0.0, lse2_p = 0.0;
     int amax = -1;
-    bool nonfinite = false, accept = true;
+    bool dbad = false, tbad = false, accept = true;  // non-finite draft row / target row at this lane's position
+    bool any_dbad = false;
 
     if (!status) {
         // Partials are merged in fp32 with the same branch-free rules the sweep uses; the draft and
@@ -831,7 +839,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             const float m = ad.x, cnt = ad.y, Zx = ad.z, S = ad.w;
             const float Z = cnt + Zx;
             if (!(cnt >= 1.f) || !(Z < 3e38f) || !(m > kFloor)) {
-                nonfinite = true;
+                dbad = true;
             } else {
                 const float lnZ = (cnt == 1.f) ? log1pf(Zx) : logf(cnt) + log1pf(Zx / cnt);
                 const float rZ = 1.f / Z;
@@ -843,20 +851,19 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         if (tg_on) {
             if (greedy) {
                 const int bi = __float_as_int(at.y);
-                if (at.z != 0.f || bi == 0x7fffffff || !(at.x > kFloor)) nonfinite = true;
+                if (at.z != 0.f || bi == 0x7fffffff || !(at.x > kFloor)) tbad = true;
                 amax = bi;
             } else {
-                if (!(at.y > 0.f) || !(at.y < 3e38f)) nonfinite = true;
+                if (!(at.y > 0.f) || !(at.y < 3e38f)) tbad = true;
                 else lse2_p = static_cast<double>(at.x) + log2_split(static_cast<double>(at.y));
             }
         }
-        if (__any_sync(0xffffffffu, nonfinite)) status |= 4;
-        if (__any_sync(0xffffffffu, badtok)) status |= 2;
+        any_dbad = __any_sync(0xffffffffu, dbad);
     }
 
     // Acceptance first: the resample kernel waits for this row's stop position, nothing waits for
     // the signals and the controller, which follow the completion flag.
-    if (status == 0 && tok_on) {
+    if (status == 0 && !any_dbad && tok_on && !badtok && !tbad) {
         if (greedy) {
             accept = (x == amax);
         } else {
@@ -867,8 +874,18 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             accept = (l2u + lq) < lp;
         }
     }
-    const unsigned rej = __ballot_sync(0xffffffffu, !accept && lane < gam);  // first rejected position
-    const int n = (status == 0 && verify) ? (rej ? (__ffs(rej) - 1) : gam) : 0;
+    // The positions are walked in order; the walk ends at the first one whose target row is non-finite
+    // (which flags the row), whose draft token is out of range, or whose token is rejected.  Target rows
+    // behind that position are not part of the step (Sec. 3.1 discards what follows the first mismatch):
+    // whatever they hold flags nothing.  A non-finite draft row flags the row wherever it is.
+    const unsigned stop = __ballot_sync(0xffffffffu, tg_on && (tbad || (lane < gam && (badtok || !accept))));
+    const int first = stop ? (__ffs(stop) - 1) : gam;
+    const bool tbad_first = __shfl_sync(0xffffffffu, tbad ? 1 : 0, first & 31) != 0;
+    if (status == 0) {
+        if (any_dbad || (verify && tbad_first)) status |= 4;
+        if (__any_sync(0xffffffffu, badtok)) status |= 2;
+    }
+    const int n = (status == 0 && verify) ? first : 0;
 
     const int rs_mode = (verify && status == 0 && !greedy) ? (n < gam ? RS_RESIDUAL : RS_BONUS) : RS_NONE;
     if (verify) {
@@ -1478,11 +1495,17 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     int mode, n;
     int4 lo4, hi4;
     if (P.rdone) {
-        if (threadIdx.x == 0) sh_flag = row_done_wait(P.rdone + b);
+        if (threadIdx.x == 0) sh_flag = row_done_wait(P.rdone + b, P.wait_limit);
         __syncthreads();
         const int v = sh_flag;
         if (!v) {
-            if (threadIdx.x == 0 && share == 0 && P.status) atomicOr(P.status + b, 16);
+            // Gave up.  The mark goes on the row's flag: if the row epilogue has already written the
+            // status (the flag went up just after the last poll) the bit is added here, otherwise the
+            // epilogue finds the mark when it raises the flag and adds the bit itself.
+            if (threadIdx.x == 0 && share == 0) {
+                const int old = atomicOr(P.rdone + b, kRowDoneTimeout);
+                if ((old & 1) && P.status) atomicOr(P.status + b, 16);
+            }
             return;
         }
         __syncthreads();  // sh_flag is reused below
@@ -1494,7 +1517,7 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
             n = lo4.y;
         } else {
             mode = (v >> 8) & 3;
-            n = v >> 16;
+            n = (v >> 16) & 0xff;
         }
     } else {
         asm volatile("griddepcontrol.wait;" ::: "memory");

@@ -37,12 +37,12 @@ def oracle_batch(s: dict, rows=None, entropy_in_bits=False, n_threads=8, tempera
                         uniforms=g("uniforms"), entropy_in_bits=entropy_in_bits, n_threads=n_threads)
 
 
-def gpu_batch(s: dict, entropy_in_bits=False, temperature_scalar=None) -> speckv.Batch:
+def gpu_batch(s: dict, entropy_in_bits=False, temperature_scalar=None, flags=0) -> speckv.Batch:
     return speckv.Batch(draft_logits=s["draft"], target_logits=s.get("target"),
                         draft_tokens=s.get("draft_tokens"), gamma=s.get("gamma"),
                         temperature=s.get("temperature"),
                         temperature_scalar=1.0 if temperature_scalar is None else temperature_scalar,
-                        uniforms=s.get("uniforms"), entropy_in_bits=entropy_in_bits)
+                        uniforms=s.get("uniforms"), entropy_in_bits=entropy_in_bits, flags=flags)
 
 
 def mlp_pair(w: dict, **kw):

@@ -281,13 +281,13 @@ def _small(dtype="fp32", B=6, G=3, V=600, seed=0):
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_row_status_flags(dtype):
     w, s = _small(dtype, B=8)
-    s["target"][1, 2, 17] = float("nan")
+    s["target"][1, 0, 17] = float("nan")       # position 0 is read whatever happens behind it
     s["draft"][2, 0, 5] = float("inf")
     s["draft"][3, 1, :] = float("-inf")
     s["draft_tokens"][4, 1] = w.V
     s["gamma"][5] = 0
     s["temperature"][6] = -1.0
-    s["target"][7, 3, :] = float("-inf")
+    s["target"][7, 0, :] = float("-inf")
     gm, om = mlp_pair(synth.make_mlp(w, DEV))
     out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
     ref = oracle.step(oracle_batch(s), s["comp"].cpu().numpy(), om)
@@ -296,6 +296,20 @@ def test_row_status_flags(dtype):
     o = {k: v.cpu().numpy() for k, v in out.items()}
     assert np.all(o["n_accepted"][1:] == 0) and np.all(o["out_tokens"][1:] == -1)
     assert np.all(o["gamma_next"][1:] == 0) and np.all(o["H"][1:] == 0) and np.all(o["scores"][1:] == 0)
+    # target rows behind the stop position are not part of the step (Sec. 3.1): a NaN there flags nothing,
+    # a NaN at the stop position does
+    n0 = int(ref["n_accepted"][0])
+    if n0 < w.gamma_max:
+        s["target"][0, n0 + 1:, 3] = float("nan")
+        out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
+        ref2 = oracle.step(oracle_batch(s), s["comp"].cpu().numpy(), om)
+        assert ref2["row_status"][0] == 0 and ref2["n_accepted"][0] == n0
+        compare_step(out, ref2)
+    s["target"][0, n0, 3] = float("nan")
+    out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
+    ref3 = oracle.step(oracle_batch(s), s["comp"].cpu().numpy(), om)
+    assert ref3["row_status"][0] == 4
+    compare_step(out, ref3)
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
