@@ -290,11 +290,21 @@ cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged
 // The stream kernel: one persistent CTA per SM (speckv_stream.cuh).
 template <typename T>
 cudaError_t launch_stream(const KParams& P, const SParams& S, cudaStream_t st, const Events& ev) {
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool slot = dev >= 0 && dev < 64;
+    if (!slot || !configured[dev].load(std::memory_order_acquire)) {
+        e = cudaFuncSetAttribute(stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSDynBytes);
+        if (e != cudaSuccess) return e;
+        if (slot) configured[dev].store(true, std::memory_order_release);
+    }
     int sms = 0;
-    cudaError_t e = sm_count(&sms);
+    e = sm_count(&sms);
     if (e != cudaSuccess) return e;
     if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
-    stream_kernel<T><<<sms, kSThreads, 0, st>>>(P, S);
+    stream_kernel<T><<<sms, kSThreads, kSDynBytes, st>>>(P, S);
     e = cudaGetLastError();
     if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
     if (ev.after_resample) cudaEventRecord(ev.after_resample, st);

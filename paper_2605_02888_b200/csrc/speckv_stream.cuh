@@ -28,15 +28,16 @@
 #pragma once
 
 #include "speckv_kernels.cuh"
+#include "speckv_pipeline.cuh"
 
 namespace speckv {
 
 constexpr int kSWarps = 32;                   // warps per CTA; one CTA per SM
 constexpr int kSThreads = kSWarps * 32;
 constexpr int kSSteps = 16;                   // vector steps (kChunk elements each) per warp quantum
-constexpr int kSU = 4;                        // loads in flight per lane
 constexpr int kSQElems = kSSteps * kChunk;    // elements per warp quantum
-constexpr int kSRing = 4;                     // items queued per CTA
+constexpr int kSRing = 8;                     // items queued per CTA
+constexpr int kSFillBatch = 4;                // stream items taken per fill at most
 constexpr int kSMaxQ = 64;                    // warp quanta per item at most
 constexpr int kSMaxB = 4096;                  // batch rows the per-CTA tables hold
 constexpr int kSMaxSlice = 16;                // slices per logit row at most
@@ -108,9 +109,9 @@ struct SItem {
     int path;      // PATH_* (sweep)
     int b, p;
     int n_q;       // warp quanta of the item
-    int Q0;        // number of its first quantum in the CTA's sequence
     int done;      // quanta finished
-    int passed;    // warps that have walked past the item
+    int busy;      // 1 from the fill until the item's last quantum has been merged; the slot is refilled after that
+    int absent;    // a quantum of a target row was left out behind a known rejection
     float scale;
     int pair;      // b*(G+1)+p
     int part_idx;  // where the item's partial goes
@@ -118,11 +119,27 @@ struct SItem {
     int elem0, n_elem;  // slice of the logit row (sweep); chunk range c0, c1 (resample)
     int rs_mode;
     float Tf;      // the batch row's temperature
+    unsigned long long ctr;  // (item's sequence number << 32) | (its quanta << 16) | quanta handed out: one atomic add
+                             // claims a quantum and tells whose it is, whatever has happened to the slot meanwhile
     const void* row;    // sweep: the logit row; resample: the target row of the stop position
     const void* drow;   // resample: the draft row of the stop position
     RowInfo ri;         // resample: the row's constants
     float4 part[kSMaxQ];
 };
+
+// Bookkeeping that needs global round trips (publishing an item's partial and taking the pair's ticket,
+// with the position epilogue behind it; the token search of a finished draw) is not done by the warp that
+// found it due: that warp is the last of its item, so already behind, and everybody else's progress is
+// bounded by the slowest warp.  It leaves a job in this queue instead, and warps that are ahead of the
+// ring and have nothing to sweep take the jobs.
+struct SJob {
+    float4 merged;
+    int type;      // 1 publish a partial, 2 search a finished draw
+    int b, p, part_idx, pair, pair_total;
+    float Tf;
+    int ready;     // 0: free; job number + 1 once the entry is written
+};
+constexpr int kSJobs = 32;
 
 struct SShared {
     int tail;        // items filled so far
@@ -131,89 +148,168 @@ struct SShared {
     int stream_done; // the global item counter has run out
     int error;
     int n_items;     // items of the whole stream
-    int q_next;      // sequence number of the next item's first quantum
     int idle_polls;
     int first_taken; // the CTA's first item is its own index in the stream, no counter involved
+    int pend_share;  // a share number taken before its row was queued; -1: none
     int n_blk;
     int phase0[kSMaxPhase + 2];
     unsigned short pre[kSMaxPhase][kSMaxB / 32 + 1];
     unsigned char gam[kSMaxB];
+    int job_head, job_tail;
+    SJob jobs[kSJobs];
     SItem ring[kSRing];
 };
 
 
 // ---- one warp quantum ---------------------------------------------------------------------------------
-// Vector step `step` of a quantum that starts at `base` and has n_valid elements (a multiple of the
-// 16-byte granule: the rows this kernel takes are 16-byte aligned and a whole number of granules long).
-// Steps beyond the end read as -inf, which no path counts.
+// The bytes in flight live in shared memory, not in registers: every lane copies its own 16-byte pieces
+// with cp.async into a ring of slots private to its warp and reads the same pieces back when their
+// group has landed, so no lane ever waits for another lane's copy and nothing needs a barrier.  A warp
+// keeps kInFlight vector steps (5.5 KB) on their way, across quantum boundaries, and they keep coming
+// in while the warp does bookkeeping.
+template <typename T> struct SStage {
+    static constexpr int kSlots = sizeof(T) == 2 ? 12 : 6;   // vector steps the warp's ring holds
+    static constexpr int kInFlight = kSlots - 1;             // a slot is refilled one step after it was read
+    static constexpr int kSlotBytes = 32 * kVec * sizeof(T);
+    static constexpr int kWarpBytes = kSlots * kSlotBytes;
+};
+constexpr int kSDynBytes = kSWarps * SStage<float>::kWarpBytes;
+static_assert(SStage<float>::kWarpBytes == SStage<__nv_bfloat16>::kWarpBytes, "one dynamic size for both types");
+
+__device__ __forceinline__ void cp_async16(uint32_t saddr, const void* g) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");
+    return v;
+}
+
+// Vector step `step` of an item that starts at `base` and has n_valid elements (a multiple of the
+// 16-byte granule: the rows this kernel takes are 16-byte aligned and a whole number of granules long)
+// goes into ring slot `slot` of the warp whose ring starts at shared address `ring`.  Pieces beyond
+// the end are not copied; sq_read gives -inf for them, which no path counts.
+//
+// Which steps make up a quantum: quantum q of an item of n_q quanta takes the item's steps q, q + n_q,
+// q + 2 n_q, ...  The warps of a CTA work on the quanta of one item at about the same pace, so what
+// they request at any moment is one contiguous stretch of the logit row (32 warps x 512 bytes), and
+// DRAM sees long sequential bursts instead of thousands of interleaved 512-byte streams.
 template <typename T>
-__device__ __forceinline__ Raw<T> sq_load(const T* base, int step, int n_valid, int lane) {
+__device__ __forceinline__ void sq_issue(uint32_t ring, int slot, const T* base, int step, int n_valid, int lane) {
+    const int e = step * kChunk + lane * kVec;  // `step` counts the item's vector steps
+    const uint32_t at = ring + slot * SStage<T>::kSlotBytes + lane * 16;
+    if constexpr (sizeof(T) == 2) {
+        if (e + kVec <= n_valid) cp_async16(at, base + e);
+    } else {
+        if (e + 4 <= n_valid) cp_async16(at, base + e);
+        if (e + 8 <= n_valid) cp_async16(at + 512, base + e + 4);
+    }
+}
+template <typename T>
+__device__ __forceinline__ Raw<T> sq_read(uint32_t ring, int slot, int step, int n_valid, int lane) {
     const int e = step * kChunk + lane * kVec;
+    const uint32_t at = ring + slot * SStage<T>::kSlotBytes + lane * 16;
     const uint32_t ninf = 0xff800000u;
     Raw<T> r;
     if constexpr (sizeof(T) == 2) {
-        if (e + kVec <= n_valid) r.a = ldg_stream(base + e);
+        if (e + kVec <= n_valid) r.a = lds128(at);
         else r.a = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
     } else {
-        if (e + 4 <= n_valid) r.a = ldg_stream(base + e);
+        if (e + 4 <= n_valid) r.a = lds128(at);
         else r.a = make_uint4(ninf, ninf, ninf, ninf);
-        if (e + 8 <= n_valid) r.b = ldg_stream(base + e + 4);
+        if (e + 8 <= n_valid) r.b = lds128(at + 512);
         else r.b = make_uint4(ninf, ninf, ninf, ninf);
     }
     return r;
 }
+template <typename T> __device__ __forceinline__ int sq_next_slot(int s) { return s + 1 == SStage<T>::kSlots ? 0 : s + 1; }
+
+// The first kInFlight steps of a quantum go out (a warp that could not chain from its previous quantum).
 template <typename T>
-__device__ __forceinline__ Raw<T> sq_pad() {
-    const uint32_t ninf = 0xff800000u;
-    Raw<T> r;
-    if constexpr (sizeof(T) == 2) {
-        r.a = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
-    } else {
-        r.a = make_uint4(ninf, ninf, ninf, ninf);
-        r.b = r.a;
+__device__ __forceinline__ void sq_prime(uint32_t ring, int& wslot, const T* base, int q, int nq, int n_valid, int lane) {
+#pragma unroll
+    for (int k = 0; k < SStage<T>::kInFlight; ++k) {
+        sq_issue<T>(ring, wslot, base, q + k * nq, n_valid, lane);
+        cp_commit();
+        wslot = sq_next_slot<T>(wslot);
     }
-    return r;
 }
 
-// Sweeps one quantum.  On entry buf holds its first kSU steps; on exit it holds the first kSU steps of
-// the quantum at nbase (n_next valid elements; nbase == nullptr: none).  e_row = index of the quantum's
-// first element within its logit row (the argmax path reports row indices).  Returns the warp's merged
-// partial in every lane.
+// Sweeps one quantum whose first kInFlight steps are on their way (or here); rslot = the slot of its
+// step 0, wslot = the slot the next copy goes to.  While it runs, the first kInFlight steps of the
+// quantum qn of the item at nbase (n_next valid elements; nbase == nullptr: none) are requested.  e_row =
+// index of the item's first element within its logit row (the argmax path reports row indices).  Returns the
+// warp's merged partial in every lane.
+//
+// The running maximum is the same in all lanes of the warp (one warp-wide maximum per vector step), so
+// a new maximum is handled by all lanes together, elements equal to it are counted by the lanes that
+// hold them, and the lanes' sums add up without any rescaling at the end of the quantum.  What a
+// quantum returns depends on its own elements only, whichever warp sweeps it and whenever.
+// (Not inlined: the loop below gets the whole register budget to itself, and what the caller keeps
+// across the call is saved once per quantum instead of spilling inside the loop.  The caller advances
+// its two slot numbers by the kSSteps steps a call consumes and issues.)
 template <typename T, int PATH>
-__device__ __forceinline__ float4 sq_sweep(const T* base, int n_valid, int e_row, float scale, Raw<T> (&buf)[kSU],
-                                           const T* nbase, int n_next) {
+__device__ __noinline__ float4 sq_sweep(uint32_t ring, int rslot, int wslot, const T* base, int q, int nq, int n_valid,
+                                        int e_row, float scale, const T* nbase, int qn, int nqn, int n_next) {
+    constexpr int F = SStage<T>::kInFlight;
     const int lane = threadIdx.x & 31;
-    // warm start: the warp-wide maximum of what is already here
-    float m0 = kFloor;
+    PipeState st;
+    st.init(scale);
+    if constexpr (PATH != PATH_ARGMAX) {
+        // start from the largest finite element of the first steps (they are read again below): fewer new
+        // maxima on the way
+        constexpr int kWarm = F < 4 ? F : 4;
+        cp_wait<F - kWarm>();
+        float m0 = kFloor;
+        int sl = rslot;
 #pragma unroll
-    for (int k = 0; k < kSU; ++k) {
-        const float v = raw_max(buf[k]);
-        if (v >= kFloor && v < __int_as_float(0x7f800000)) m0 = fmaxf(m0, v);
+        for (int k = 0; k < kWarm; ++k) {
+            const float v = raw_max(sq_read<T>(ring, sl, q + k * nq, n_valid, lane));
+            if (v >= kFloor && v < __int_as_float(0x7f800000)) m0 = fmaxf(m0, v);
+            sl = sq_next_slot<T>(sl);
+        }
+        m0 = warp_maxf(m0);
+        st.M = m0;
+        st.r = m0 * scale;
     }
-    m0 = warp_maxf(m0);
-    DraftState ds; TargetState ts; ArgmaxState as;
-    if constexpr (PATH == PATH_DRAFT) ds.init(m0);
-    else if constexpr (PATH == PATH_TARGET) ts.init(m0, scale);
-    else as.init(m0);
-#pragma unroll
-    for (int batch = 0; batch < kSSteps / kSU; ++batch) {
-#pragma unroll
-        for (int k = 0; k < kSU; ++k) {
-            const Raw<T> cur = buf[k];
-            const int step = batch * kSU + k;
-            if (batch + 1 < kSSteps / kSU) buf[k] = sq_load<T>(base, step + kSU, n_valid, lane);
-            else if (nbase) buf[k] = sq_load<T>(nbase, k, n_next, lane);
-            else buf[k] = sq_pad<T>();
-            if constexpr (PATH == PATH_DRAFT) ds.template step<T>(cur, scale);
-            else if constexpr (PATH == PATH_TARGET) ts.template step<T>(cur, scale);
-            else as.template step<T>(cur, e_row + step * kChunk + lane * kVec);
+    const f2 sc2 = pack2(scale, scale);
+    // (a short loop body: every warp of the SM runs this loop at its own place, and what they run has to
+    // stay in the instruction cache)
+#pragma unroll 2
+    for (int step = 0; step < kSSteps; ++step) {
+        cp_wait<F - 1>();
+        const Raw<T> cur = sq_read<T>(ring, rslot, q + step * nq, n_valid, lane);
+        rslot = sq_next_slot<T>(rslot);
+        if (step + F < kSSteps) sq_issue<T>(ring, wslot, base, q + (step + F) * nq, n_valid, lane);
+        else if (nbase) sq_issue<T>(ring, wslot, nbase, qn + (step + F - kSSteps) * nqn, n_next, lane);
+        cp_commit();
+        wslot = sq_next_slot<T>(wslot);
+        if constexpr (PATH == PATH_ARGMAX) {
+            st.as.template step<T>(cur, e_row + (q + step * nq) * kChunk + lane * kVec);
+        } else {
+            const float um = raw_max(cur);
+            const float wm = warp_max_nan(um);  // NaN wins
+            if (!(wm < __int_as_float(0x7f800000))) {
+                st.bad = true;  // NaN or +inf: the row gets flagged
+            } else if constexpr (PATH == PATH_DRAFT) {
+                if (wm > st.M) draft_rescale(st, wm, scale);
+                if (__any_sync(0xffffffffu, um == st.M)) draft_unit_careful<T>(st, cur, scale);
+                else draft_unit_fast<T>(st, cur, pack2(st.M, st.M), sc2);
+            } else {
+                if (wm > st.M) target_rescale(st, wm, scale);
+                target_unit<T>(st, cur, sc2, pack2(-st.r, -st.r));
+            }
         }
     }
-    float4 part;
-    if constexpr (PATH == PATH_DRAFT) part = ds.partial();
-    else if constexpr (PATH == PATH_TARGET) part = ts.partial();
-    else part = as.partial();
-    return warp_merge<PATH>(part, scale);
+    const float nan = __int_as_float(0x7fc00000);
+    if constexpr (PATH == PATH_DRAFT)
+        return make_float4(st.M, warp_sumf(st.bad ? nan : st.cnt), warp_sumf(st.zsum()), warp_sumf(st.ssum()));
+    else if constexpr (PATH == PATH_TARGET)
+        return make_float4(st.r, warp_sumf(st.bad ? nan : st.zsum()), 0.f, 0.f);
+    else
+        return warp_merge<PATH_ARGMAX>(st.as.partial(), scale);
 }
 
 __device__ __forceinline__ float4 s_neutral(int path) {
@@ -531,6 +627,7 @@ template <typename T>
 __device__ __noinline__ void s_search(const KParams& P, const SParams& S, int b, int gam, const RowInfo& ri,
                                       const T* trow, const T* drow) {
     const int lane = threadIdx.x & 31;
+    __threadfence();
     RsConst c = rs_const(ri, ri.mode);
     float* csum = P.csum + static_cast<long long>(b) * P.nchunk;
     const int per_lane = (P.nchunk + 31) / 32;
@@ -596,10 +693,10 @@ __device__ __forceinline__ void s_decode(const KParams& P, const SParams& S, con
     slot = r - __shfl_sync(0xffffffffu, before, j);
 }
 
-// Item `seq` finished its last quantum on this warp: one partial per (logit row, slice) goes out, the
-// pair's ticket is taken, and the warp that completes the pair runs the position's epilogue.
+// One partial per (logit row, slice) goes out, the pair's ticket is taken, and the warp that completes the
+// pair runs the position's epilogue.
 template <typename T>
-__device__ __forceinline__ void s_publish(const KParams& P, const SParams& S, const SShared& sh, float4 merged, int b, int p,
+__device__ __noinline__ void s_publish(const KParams& P, const SParams& S, const SShared& sh, float4 merged, int b, int p,
                                           int part_idx, int pair, int pair_total, float Tf) {
     const int lane = threadIdx.x & 31;
     int t = 0;
@@ -613,6 +710,77 @@ __device__ __forceinline__ void s_publish(const KParams& P, const SParams& S, co
         __threadfence();
         s_pair_epilogue<T>(P, S, b, p, sh.gam[b], Tf);
     }
+}
+
+template <typename T>
+__device__ __noinline__ void s_do_job(const KParams& P, const SParams& S, SShared& sh, const SJob& j) {
+    if (j.type == 1) {
+        s_publish<T>(P, S, sh, j.merged, j.b, j.p, j.part_idx, j.pair, j.pair_total, j.Tf);
+    } else {
+        const int4* ip = reinterpret_cast<const int4*>(P.info + j.b);
+        const RowInfo ri = row_info_from(__ldcg(ip), __ldcg(ip + 1));
+        const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(j.b) * P.tsb + static_cast<long long>(ri.n) * P.tsp;
+        const T* drow = static_cast<const T*>(P.d) + static_cast<long long>(j.b) * P.dsb + static_cast<long long>(ri.n) * P.dsp;
+        s_search<T>(P, S, j.b, sh.gam[j.b], ri, trow, drow);
+    }
+}
+
+// Leave a job in the queue (whole warp calls; every lane holds the same job).  When the entry it would go
+// to is still occupied the caller does the job itself.
+template <typename T>
+__device__ __forceinline__ void s_job_push(const KParams& P, const SParams& S, SShared& sh, const SJob& j) {
+    const int lane = threadIdx.x & 31;
+    int at = -1;
+    if (lane == 0) {
+        for (;;) {
+            const int t = s_vol(&sh.job_tail);
+            if (s_vol(&sh.jobs[t % kSJobs].ready) != 0) break;  // the entry of 32 jobs ago has not been taken yet
+            if (atomicCAS(&sh.job_tail, t, t + 1) == t) { at = t; break; }
+        }
+        if (at >= 0) {
+            SJob* e = &sh.jobs[at % kSJobs];
+            e->merged = j.merged; e->type = j.type; e->b = j.b; e->p = j.p; e->part_idx = j.part_idx;
+            e->pair = j.pair; e->pair_total = j.pair_total; e->Tf = j.Tf;
+            __threadfence_block();
+            *reinterpret_cast<volatile int*>(&e->ready) = at + 1;
+        }
+    }
+    at = __shfl_sync(0xffffffffu, at, 0);
+    if (at < 0) s_do_job<T>(P, S, sh, j);
+}
+
+// Reserve the oldest job nobody has reserved yet: its number, or -1.  The warp that holds a number runs
+// that job (s_job_run) as soon as it has no quantum in hand.
+__device__ __forceinline__ int s_job_reserve(SShared& sh) {
+    int r = -1;
+    if ((threadIdx.x & 31) == 0) {
+        const int have = s_vol(&sh.job_head);
+        if (have < s_vol(&sh.job_tail) && atomicCAS(&sh.job_head, have, have + 1) == have) r = have;
+    }
+    return __shfl_sync(0xffffffffu, r, 0);
+}
+template <typename T>
+__device__ __forceinline__ void s_job_run(const KParams& P, const SParams& S, SShared& sh, int r) {
+    const int lane = threadIdx.x & 31;
+    SJob j;
+    if (lane == 0) {
+        SJob* e = &sh.jobs[r % kSJobs];
+        for (int k = 0; k < S.poll_limit && s_vol(&e->ready) != r + 1; ++k) {}  // being written by its pusher right now
+        __threadfence_block();
+        const volatile SJob* v = e;
+        j.merged = make_float4(v->merged.x, v->merged.y, v->merged.z, v->merged.w);
+        j.type = v->type; j.b = v->b; j.p = v->p; j.part_idx = v->part_idx; j.pair = v->pair;
+        j.pair_total = v->pair_total; j.Tf = v->Tf;
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&e->ready) = 0;  // the entry may be used again
+    }
+    j.merged.x = __shfl_sync(0xffffffffu, j.merged.x, 0); j.merged.y = __shfl_sync(0xffffffffu, j.merged.y, 0);
+    j.merged.z = __shfl_sync(0xffffffffu, j.merged.z, 0); j.merged.w = __shfl_sync(0xffffffffu, j.merged.w, 0);
+    j.type = __shfl_sync(0xffffffffu, j.type, 0); j.b = __shfl_sync(0xffffffffu, j.b, 0);
+    j.p = __shfl_sync(0xffffffffu, j.p, 0); j.part_idx = __shfl_sync(0xffffffffu, j.part_idx, 0);
+    j.pair = __shfl_sync(0xffffffffu, j.pair, 0); j.pair_total = __shfl_sync(0xffffffffu, j.pair_total, 0);
+    j.Tf = __shfl_sync(0xffffffffu, j.Tf, 0);
+    s_do_job<T>(P, S, sh, j);
 }
 
 template <typename T>
@@ -635,8 +803,13 @@ __device__ __forceinline__ void s_finish_sweep(const KParams& P, const SParams& 
     float4 v = s_neutral(path);
     if (lane < nq) v = make_float4(vp[lane].x, vp[lane].y, vp[lane].z, vp[lane].w);
     if (lane + 32 < nq) v = s_merge(path, v, make_float4(vp[lane + 32].x, vp[lane + 32].y, vp[lane + 32].z, vp[lane + 32].w), scale);
-    const float4 merged = s_warp_merge(path, v, scale);
-    s_publish<T>(P, S, sh, merged, it.b, it.p, it.part_idx, it.pair, it.pair_total, it.Tf);
+    SJob j;
+    j.merged = s_warp_merge(path, v, scale);
+    if (s_vol(&it.absent)) j.merged = make_float4(0.f, 0.f, 0.f, 1.f);  // part of the row was left out: the row counts as not read
+    j.type = 1; j.b = it.b; j.p = it.p; j.part_idx = it.part_idx; j.pair = it.pair; j.pair_total = it.pair_total; j.Tf = it.Tf;
+    __syncwarp();
+    if (lane == 0) { __threadfence_block(); *reinterpret_cast<volatile int*>(&it.busy) = 0; }  // the slot may be refilled
+    s_job_push<T>(P, S, sh, j);
 }
 
 template <typename T>
@@ -656,14 +829,17 @@ __device__ __forceinline__ void s_resample_job(const KParams& P, const SParams& 
     if (lane == 0) {
         const int d = atomicAdd(&it.done, 1);
         if (d == it.n_q - 1) {
+            *reinterpret_cast<volatile int*>(&it.busy) = 0;  // the slot may be refilled
             __threadfence();
             last = (atomicAdd(P.tick2 + b, 1) == S.rs_shares - 1);
         }
     }
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) {
-        __threadfence();
-        s_search<T>(P, S, b, sh.gam[b], ri, trow, drow);
+        SJob j;
+        j.merged = make_float4(0.f, 0.f, 0.f, 0.f);
+        j.type = 2; j.b = b; j.p = 0; j.part_idx = 0; j.pair = 0; j.pair_total = 0; j.Tf = 0.f;
+        s_job_push<T>(P, S, sh, j);
     }
 }
 
@@ -677,35 +853,42 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
     int got = 0;
     if (lane == 0) got = (atomicCAS(&sh.lock, 0, 1) == 0);
     got = __shfl_sync(0xffffffffu, got, 0);
-    if (!got) { if (starving) __nanosleep(200); return; }
+    if (!got) { if (starving) __nanosleep(1500); return; }
     auto unlock = [&]() {
         __syncwarp();
         if (lane == 0) { __threadfence_block(); atomicExch(&sh.lock, 0); }
     };
     const int tail = s_vol(&sh.tail);
     SItem& it = sh.ring[tail % kSRing];
-    const bool slot_free = tail < kSRing || s_vol(&it.passed) == kSWarps;
-    if (!slot_free || s_vol(&sh.exhausted)) { unlock(); if (starving) __nanosleep(100); return; }
+    const bool slot_free = tail < kSRing || s_vol(&it.busy) == 0;
+    if (!slot_free || s_vol(&sh.exhausted)) { unlock(); if (starving) __nanosleep(1500); return; }
 
-    // 1. a share of a queued draw
-    int share = -1;
+    // A share of a queued draw comes first (its rows are the freshest in L2).  The counter is a plain
+    // atomic add, so nobody retries; a share number beyond the rows queued so far (another CTA was quicker)
+    // is kept until its row arrives.
+    int share = -1, brow = -1;
     if (lane == 0) {
-        const int nx = ld_relaxed(&S.ctrl->rs_next);
-        const int tq = ld_relaxed(&S.ctrl->rs_tail);
-        if (nx < tq * S.rs_shares) share = (atomicCAS(&S.ctrl->rs_next, nx, nx + 1) == nx) ? nx : -2;
+        share = sh.pend_share;
+        if (share < 0) {
+            const int nx = ld_relaxed(&S.ctrl->rs_next);
+            const int tq = ld_relaxed(&S.ctrl->rs_tail);
+            if (nx < tq * S.rs_shares) share = atomicAdd(&S.ctrl->rs_next, 1);
+        }
+        int v = 0;
+        if (share >= 0) {
+            const int qpos = share / S.rs_shares;
+            if (qpos >= P.B) share = -1;                 // beyond anything that can ever be queued
+            else v = ld_acquire(S.rsq + qpos);
+        }
+        if (share >= 0 && v == 0) { sh.pend_share = share; share = -1; }
+        else sh.pend_share = -1;
+        brow = v - 1;
     }
     share = __shfl_sync(0xffffffffu, share, 0);
-    if (share == -2) { unlock(); return; }
+    brow = __shfl_sync(0xffffffffu, brow, 0);
     if (share >= 0) {
-        const int qpos = share / S.rs_shares, part = share - qpos * S.rs_shares;
-        int v = 0;
-        if (lane == 0) {
-            for (int k = 0; k < S.poll_limit && v == 0; ++k) v = ld_acquire(S.rsq + qpos);  // written right after the tail moved
-            if (v == 0) { sh.error = 1; sh.exhausted = 1; }
-        }
-        v = __shfl_sync(0xffffffffu, v, 0);
-        if (v == 0) { unlock(); return; }
-        const int b = v - 1;
+        const int part = share % S.rs_shares;
+        const int b = brow;
         if (lane == 0) {
             const int4* ip = reinterpret_cast<const int4*>(P.info + b);
             const RowInfo ri = row_info_from(__ldcg(ip), __ldcg(ip + 1));
@@ -713,67 +896,14 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
             it.elem0 = part * kSRsShare;
             it.n_elem = min(P.nchunk, it.elem0 + kSRsShare);
             it.n_q = (it.n_elem - it.elem0 + kSRsSub - 1) / kSRsSub;
-            it.Q0 = sh.q_next; sh.q_next += it.n_q;
-            it.done = 0; it.passed = 0;
+            it.done = 0; it.busy = 1; it.absent = 0;
             it.ri = ri;
             it.row = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(ri.n) * P.tsp;
             it.drow = static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb + static_cast<long long>(ri.n) * P.dsp;
             sh.idle_polls = 0;
             __threadfence_block();
-            *reinterpret_cast<volatile int*>(&sh.tail) = tail + 1;
-        }
-        unlock();
-        return;
-    }
-
-    // 2. the next item of the stream
-    if (!s_vol(&sh.stream_done)) {
-        int i = 0;
-        if (lane == 0) {
-            if (!sh.first_taken) { sh.first_taken = 1; i = blockIdx.x; }
-            else i = static_cast<int>(gridDim.x) + atomicAdd(&S.ctrl->item_next, 1);
-        }
-        i = __shfl_sync(0xffffffffu, i, 0);
-        if (i >= sh.n_items) {
-            if (lane == 0) sh.stream_done = 1;
-            unlock();
-            return;
-        }
-        int b, p, slot, slice;
-        s_decode(P, S, sh, i, b, p, slot, slice);
-        const int gam = sh.gam[b];
-        const float Tf = P.temp ? __ldg(P.temp + b) : P.temp_scalar;
-        // a target row behind a known rejection is not part of the step (Sec. 3.1)
-        bool skip = false;
-        if (slot == 0 && p >= 1 && !S.read_all) {
-            const unsigned long long st = ld_state(S.state + b);
-            skip = ((st >> kStRej) & ((1ull << p) - 1ull)) != 0;
-        }
-        const bool greedy = (Tf == 0.f);
-        const int pair = b * (P.G + 1) + p;
-        const int part_idx = (pair * 2 + slot) * S.n_slice + slice;
-        const int pair_total = S.n_slice * (p < gam ? 2 : 1);
-        if (skip) {
-            unlock();
-            s_publish<T>(P, S, sh, make_float4(0.f, 0.f, 0.f, 1.f), b, p, part_idx, pair, pair_total, Tf);
-            return;
-        }
-        if (lane == 0) {
-            it.type = 1;
-            it.path = slot == 1 ? PATH_DRAFT : (greedy ? PATH_ARGMAX : PATH_TARGET);
-            it.b = b; it.p = p;
-            it.elem0 = slice * S.slice_elems;
-            it.n_elem = min(P.V - it.elem0, S.slice_elems);
-            it.n_q = (it.n_elem + kSQElems - 1) / kSQElems;
-            it.Q0 = sh.q_next; sh.q_next += it.n_q;
-            it.done = 0; it.passed = 0;
-            it.scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
-            it.Tf = Tf;
-            it.pair = pair; it.part_idx = part_idx; it.pair_total = pair_total;
-            it.row = slot == 1
-                ? static_cast<const void*>(static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb + static_cast<long long>(p) * P.dsp)
-                : static_cast<const void*>(static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(p) * P.tsp);
-            sh.idle_polls = 0;
+            *reinterpret_cast<volatile unsigned long long*>(&it.ctr) =
+                (static_cast<unsigned long long>(tail) << 32) | (static_cast<unsigned long long>(it.n_q) << 16);
             __threadfence_block();
             *reinterpret_cast<volatile int*>(&sh.tail) = tail + 1;
         }
@@ -781,32 +911,120 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
         return;
     }
 
-    // 3. nothing to hand out: done once every batch row has its outputs
+    // The stream's next items: as many as there are free slots in a row (at most kSFillBatch) for one
+    // atomic add, so that a fill's global round trips are shared by several items.
+    if (!s_vol(&sh.stream_done)) {
+        int i0 = -1, k = 0;
+        if (lane == 0) {
+            int kfree = 1;
+            while (kfree < kSFillBatch && (tail + kfree < kSRing || s_vol(&sh.ring[(tail + kfree) % kSRing].busy) == 0)) ++kfree;
+            if (!sh.first_taken) { sh.first_taken = 1; i0 = blockIdx.x; k = 1; }
+            else { k = kfree; i0 = static_cast<int>(gridDim.x) + atomicAdd(&S.ctrl->item_next, k); }
+            if (i0 >= sh.n_items) k = 0;
+            else if (i0 + k > sh.n_items) k = sh.n_items - i0;
+            if (i0 + k >= sh.n_items) sh.stream_done = 1;
+        }
+        i0 = __shfl_sync(0xffffffffu, i0, 0);
+        k = __shfl_sync(0xffffffffu, k, 0);
+        if (k > 0) {
+            int bb[kSFillBatch], pp[kSFillBatch], sl[kSFillBatch], sc[kSFillBatch];
+            float Tfs[kSFillBatch];
+#pragma unroll
+            for (int j = 0; j < kSFillBatch; ++j) {
+                bb[j] = 0; pp[j] = 0; sl[j] = 0; sc[j] = 0; Tfs[j] = 1.f;
+                if (j < k) {
+                    s_decode(P, S, sh, i0 + j, bb[j], pp[j], sl[j], sc[j]);
+                    Tfs[j] = P.temp ? __ldg(P.temp + bb[j]) : P.temp_scalar;
+                }
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int j = 0; j < kSFillBatch; ++j) {
+                    if (j >= k) break;
+                    SItem& x = sh.ring[(tail + j) % kSRing];
+                    const int b = bb[j], p = pp[j], slot = sl[j], slice = sc[j];
+                    const float Tf = Tfs[j];
+                    const bool greedy = (Tf == 0.f);
+                    x.type = 1;
+                    x.path = slot == 1 ? PATH_DRAFT : (greedy ? PATH_ARGMAX : PATH_TARGET);
+                    x.b = b; x.p = p;
+                    x.elem0 = slice * S.slice_elems;
+                    x.n_elem = min(P.V - x.elem0, S.slice_elems);
+                    x.n_q = (x.n_elem + kSQElems - 1) / kSQElems;
+                    x.done = 0; x.busy = 1; x.absent = 0;
+                    x.scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
+                    x.Tf = Tf;
+                    x.pair = b * (P.G + 1) + p;
+                    x.part_idx = (x.pair * 2 + slot) * S.n_slice + slice;
+                    x.pair_total = S.n_slice * (p < sh.gam[b] ? 2 : 1);
+                    x.row = slot == 1
+                        ? static_cast<const void*>(static_cast<const T*>(P.d) + static_cast<long long>(b) * P.dsb + static_cast<long long>(p) * P.dsp)
+                        : static_cast<const void*>(static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(p) * P.tsp);
+                    __threadfence_block();
+                    *reinterpret_cast<volatile unsigned long long*>(&x.ctr) =
+                        (static_cast<unsigned long long>(tail + j) << 32) | (static_cast<unsigned long long>(x.n_q) << 16);
+                }
+                sh.idle_polls = 0;
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(&sh.tail) = tail + k;
+            }
+        }
+        unlock();
+        return;
+    }
+
+    // nothing to hand out: done once every batch row has its outputs
     if (lane == 0) {
         if (ld_relaxed(&S.ctrl->resolved) >= P.B) sh.exhausted = 1;
         else if (++sh.idle_polls > S.poll_limit) { sh.error = 1; sh.exhausted = 1; }
     }
     unlock();
-    if (starving) __nanosleep(300);
+    if (starving) __nanosleep(1500);
 }
 
-// Is quantum g of this warp's sequence in the ring?  Moves s_look past the items that lie before it.
-__device__ __forceinline__ bool s_lookup(const SShared& sh, int g, int& s_look, int& q) {
+// Claims the next quantum of the CTA's ring for this warp: one atomic add on the item's counter, which
+// carries the item's sequence number, so a warp whose cursor has fallen behind a refilled slot simply
+// finds itself holding a quantum of the newer item.  A quantum of a target row behind a rejection that
+// has become known since the item was filled is settled on the spot (Sec. 3.1: such a row is not part
+// of the step).  `blocking`: with nothing in the ring the warp does queued jobs, fills, or naps, until
+// there is a quantum or the step is over; otherwise it returns false at once.
+template <typename T>
+__device__ __forceinline__ bool s_claim(const KParams& P, const SParams& S, SShared& sh, int& cursor, SItem*& out_it,
+                                        int& out_q, bool blocking) {
+    const int lane = threadIdx.x & 31;
     for (;;) {
-        if (s_look >= s_vol(&sh.tail)) return false;
-        const SItem& it = sh.ring[s_look % kSRing];
-        const int q0 = s_vol(&it.Q0), nq = s_vol(&it.n_q);
-        if (g < q0 + nq) { q = g - q0; return true; }
-        ++s_look;
+        if (blocking) {  // a warp without a quantum in hand takes queued bookkeeping first
+            const int r = s_job_reserve(sh);
+            if (r >= 0) { s_job_run<T>(P, S, sh, r); continue; }
+        }
+        if (cursor >= s_vol(&sh.tail)) {
+            if (!blocking) return false;
+            if (s_vol(&sh.exhausted)) return false;
+            s_try_fill<T>(P, S, sh, true);
+            continue;
+        }
+        SItem* it = &sh.ring[cursor % kSRing];
+        unsigned long long v = 0;
+        if (lane == 0) v = atomicAdd(&it->ctr, 1ull);
+        v = __shfl_sync(0xffffffffu, v, 0);
+        const int seq = static_cast<int>(v >> 32), q = static_cast<int>(v & 0xffffu);
+        if (seq > cursor) cursor = seq;
+        if (q >= static_cast<int>((v >> 16) & 0xffffu)) { cursor = seq + 1; continue; }
+        if (it->type == 1 && it->path != PATH_DRAFT && it->p >= 1 && !S.read_all) {
+            unsigned long long st = 0;
+            if (lane == 0) st = ld_state(S.state + it->b);
+            st = __shfl_sync(0xffffffffu, st, 0);
+            if (((st >> kStRej) & ((1ull << it->p) - 1ull)) != 0) {
+                if (lane == 0) *reinterpret_cast<volatile int*>(&it->absent) = 1;
+                s_finish_sweep<T>(P, S, sh, *it, q, s_neutral(it->path));
+                continue;
+            }
+        }
+        out_it = it;
+        out_q = q;
+        return true;
     }
 }
-__device__ __forceinline__ void s_pass_upto(SShared& sh, int& s_pass, int upto) {
-    if ((threadIdx.x & 31) == 0)
-        for (int s = s_pass; s < upto; ++s) atomicAdd(&sh.ring[s % kSRing].passed, 1);
-    s_pass = upto > s_pass ? upto : s_pass;
-    __syncwarp();
-}
-
 
 // ---- the kernel -------------------------------------------------------------------------------------------
 template <typename T>
@@ -820,8 +1038,10 @@ __global__ void __launch_bounds__(kSThreads, 1) stream_kernel(const __grid_const
     const int n_blk = (P.B + 31) / 32;
     if (threadIdx.x == 0) {
         sh.tail = 0; sh.lock = 0; sh.exhausted = 0; sh.stream_done = 0; sh.error = 0;
-        sh.q_next = 0; sh.idle_polls = 0; sh.first_taken = 0; sh.n_blk = n_blk;
+        sh.idle_polls = 0; sh.first_taken = 0; sh.n_blk = n_blk;
+        sh.job_head = 0; sh.job_tail = 0; sh.pend_share = -1;
     }
+    if (threadIdx.x < kSJobs) sh.jobs[threadIdx.x].ready = 0;  // shared memory keeps what the last launch left
     for (int blk = warp; blk < n_blk; blk += kSWarps) {
         const int b = blk * 32 + lane;
         int gam = 0;
@@ -883,60 +1103,60 @@ __global__ void __launch_bounds__(kSThreads, 1) stream_kernel(const __grid_const
         }
     }
 
-    // ---- every warp walks its own sequence of quanta: g = warp, warp + 32, ... ----
-    int g = warp, s_look = 0, s_pass = 0;
-    Raw<T> buf[kSU];
-    for (;;) {
-        int q = 0;
-        bool out = false;
-        while (!s_lookup(sh, g, s_look, q)) {
-            s_pass_upto(sh, s_pass, s_look);
-            if (s_vol(&sh.exhausted)) { out = true; break; }
-            s_try_fill<T>(P, S, sh, true);
-        }
-        if (out) break;
-        SItem* it = &sh.ring[s_look % kSRing];
+    // ---- every warp: claim a quantum, sweep it (with the next one's first loads already out), post it ----
+    extern __shared__ __align__(128) unsigned char s_dyn[];
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(s_dyn)) + warp * SStage<T>::kWarpBytes;
+    int cursor = 0, rslot = 0, wslot = 0;
+    SItem* it = nullptr;
+    int q = 0;
+    bool have = s_claim<T>(P, S, sh, cursor, it, q, true);
+    while (have) {
         if (it->type == 2) {
             s_resample_job<T>(P, S, sh, *it, q);
-            g += kSWarps;
+            have = s_claim<T>(P, S, sh, cursor, it, q, true);
             continue;
         }
-        const T* base = static_cast<const T*>(it->row) + it->elem0 + q * kSQElems;
-        int n_valid = min(kSQElems, it->n_elem - q * kSQElems);
-#pragma unroll
-        for (int k = 0; k < kSU; ++k) buf[k] = sq_load<T>(base, k, n_valid, lane);
+        const T* base = static_cast<const T*>(it->row) + it->elem0;
+        int n_valid = it->n_elem, nq = it->n_q;
+        rslot = wslot;  // nothing of this warp is in flight: the ring starts afresh wherever the write slot stands
+        sq_prime<T>(ring, wslot, base, q, nq, n_valid, lane);
         for (;;) {
-            // keep the ring a few items ahead of the warps (a fill is a chain of global round trips; paid
-            // here, with this warp's loads in flight, it is hidden; paid when a warp runs dry, it is not)
-            if (s_vol(&sh.tail) - s_look < kSRing - 1 && !s_vol(&sh.lock) && !s_vol(&sh.exhausted) &&
+            // whoever passes here while the ring has a free slot fills it (a fill is a chain of global round
+            // trips; paid here, with this warp's copies in flight, it is hidden)
+            if (!s_vol(&sh.lock) && !s_vol(&sh.exhausted) &&
+                (s_vol(&sh.tail) < kSRing || s_vol(&sh.ring[s_vol(&sh.tail) % kSRing].busy) == 0) &&
                 !(s_vol(&sh.stream_done) && ld_relaxed(&S.ctrl->rs_next) >= ld_relaxed(&S.ctrl->rs_tail) * S.rs_shares))
                 s_try_fill<T>(P, S, sh, false);
-            // the quantum after this one, if its item is already in the ring: its first loads go out
-            // before this one is merged
-            int s_next = s_look, qn = 0;
-            const bool ahead = s_lookup(sh, g + kSWarps, s_next, qn);
-            SItem* nit = &sh.ring[s_next % kSRing];
+            // the quantum after this one, if the ring has one: its first copies go out while this one is swept
+            // (unless bookkeeping is queued: then this warp reserves a job and runs it after this quantum)
+            SItem* nit = nullptr;
+            int qn = 0;
+            const int job = s_job_reserve(sh);
+            const bool ahead = job < 0 && s_claim<T>(P, S, sh, cursor, nit, qn, false);
             const bool chain = ahead && nit->type == 1;
             const T* nbase = nullptr;
-            int n_next = 0;
+            int n_next = 0, nqn = 1;
             if (chain) {
-                nbase = static_cast<const T*>(nit->row) + nit->elem0 + qn * kSQElems;
-                n_next = min(kSQElems, nit->n_elem - qn * kSQElems);
+                nbase = static_cast<const T*>(nit->row) + nit->elem0;
+                n_next = nit->n_elem;
+                nqn = nit->n_q;
             }
-            const int e_row = it->elem0 + q * kSQElems;
+            const int e_row = it->elem0;
             const float scale = it->scale;
             const int path = it->path;
             float4 part;
-            if (path == PATH_DRAFT) part = sq_sweep<T, PATH_DRAFT>(base, n_valid, e_row, scale, buf, nbase, n_next);
-            else if (path == PATH_TARGET) part = sq_sweep<T, PATH_TARGET>(base, n_valid, e_row, scale, buf, nbase, n_next);
-            else part = sq_sweep<T, PATH_ARGMAX>(base, n_valid, e_row, scale, buf, nbase, n_next);
+            if (path == PATH_DRAFT) part = sq_sweep<T, PATH_DRAFT>(ring, rslot, wslot, base, q, nq, n_valid, e_row, scale, nbase, qn, nqn, n_next);
+            else if (path == PATH_TARGET) part = sq_sweep<T, PATH_TARGET>(ring, rslot, wslot, base, q, nq, n_valid, e_row, scale, nbase, qn, nqn, n_next);
+            else part = sq_sweep<T, PATH_ARGMAX>(ring, rslot, wslot, base, q, nq, n_valid, e_row, scale, nbase, qn, nqn, n_next);
+            rslot = (rslot + kSSteps) % SStage<T>::kSlots;
+            wslot = (wslot + kSSteps) % SStage<T>::kSlots;
             s_finish_sweep<T>(P, S, sh, *it, q, part);
-            g += kSWarps;
-            s_look = s_next;
-            s_pass_upto(sh, s_pass, s_look);
+            if (job >= 0) s_job_run<T>(P, S, sh, job);
+            have = ahead;
+            it = nit; q = qn; base = nbase; n_valid = n_next; nq = nqn;
             if (!chain) break;
-            it = nit; q = qn; base = nbase; n_valid = n_next;
         }
+        if (!have) have = s_claim<T>(P, S, sh, cursor, it, q, true);
     }
 
     // a poll limit ran out somewhere: the batch rows this CTA answers for and that are not complete get
