@@ -3,6 +3,10 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload b256]
 
+With --gpus N > 1 and no launcher around it (WORLD_SIZE unset) it starts the N ranks itself, one process
+per GPU on 127.0.0.1; under torchrun it is one of the ranks.  Rows never interact, so the ranks share
+nothing but the barrier and the MAX of their times.
+
 A step = one pass of the whole hot path (draft signals, controller, verification: a memset of the
 tickets, then the sweep kernel, whose grid also draws the fresh tokens for bf16 logits; for fp32
 logits the ring sweep and the resample kernel) over one synthetic batch whose logits are resident
@@ -29,7 +33,7 @@ for _p in (ROOT, os.path.join(ROOT, "tests")):
 
 METRIC = "verified_speculation_rows_per_sec"
 UNIT = "rows/s"
-FALLBACK_HBM_GBS = 6650.0  # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+FALLBACK_HBM_GBS = 6650.0  # an earlier STREAM-style copy measurement on a B200, used only if MEASURED_PEAKS.json is absent
 
 
 def _env_int(k, d):
@@ -118,6 +122,14 @@ class ClockSampler(threading.Thread):
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def config_of(w) -> dict:
+    """The workload as both arms name it."""
+    return {"workload": w.name, "B_per_gpu": w.B, "gamma_max": w.gamma_max, "V": w.V, "logits": w.dtype,
+            "temperature": w.temperature, "temperature_mode": w.temperature_mode,
+            "gamma_per_row": {"choices": "hash-uniform over {2,4,6,8}", "ragged": "hash-uniform over 1..gamma_max"}.get(
+                w.gamma_mode, f"{min(w.gamma_fixed, w.gamma_max)} for every row")}
+
+
 def run_reference(args, w):
     """The oracle as the timed arm: each step is a bounded sample of rows of the workload."""
     import numpy as np
@@ -159,12 +171,58 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "B": w.B, "gamma_max": w.gamma_max, "V": w.V, "logits": w.dtype,
-                   "rows_per_step_sampled": rows},
+        "config": config_of(w),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
+
+
+def launch_ranks(n: int, argv, extra_env=None) -> int:
+    """Start n copies of this script as ranks 0..n-1 of one job on this host and wait for them.
+    Rank 0's stdout is passed through (it prints the JSON line); returns the worst exit code."""
+    import socket
+    import subprocess
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), **(extra_env or {}))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for pr in procs:
+        rc = max(rc, abs(pr.wait()))
+    return rc
+
+
+def run_dry(args):
+    """The launcher and the rank plumbing without a GPU: gloo ranks, the row split of the sharded path,
+    the barrier and the MAX reduction of the times, and rank 0's JSON line.  No kernel runs and the line
+    carries no throughput."""
+    import torch
+    import torch.distributed as dist
+    from paper_2605_02888_b200 import shard, synth
+    world, rank = _env_int("WORLD_SIZE", 1), _env_int("RANK", 0)
+    if world > 1:
+        dist.init_process_group("gloo")
+    w = synth.WORKLOADS[args.workload]
+    rr = shard.row_range(w.B * world, rank, world)
+    lo, hi = rr.start, rr.stop
+    t = torch.tensor([float(rank + 1)])
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        rows = [None] * world
+        dist.all_gather_object(rows, (lo, hi))
+    else:
+        rows = [(lo, hi)]
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "max_over_ranks": float(t.item()), "row_ranges": rows}))
+    if world > 1:
+        dist.destroy_process_group()
 
 
 def main():
@@ -178,7 +236,24 @@ def main():
     ap.add_argument("--lib", default=None, help="path of a libspeckv.so build to load instead of the in-tree one")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-early-exit", action="store_true",
+                    help="read every target row (SPECKV_READ_ALL_TARGET_ROWS): the all-positions reference for GB/s")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "stream", "sliced"], help="kernel choice hint passed to the library")
+    ap.add_argument("--min-seconds", type=float, default=0.5, help="the timed blocks are repeated until this much time has passed")
+    ap.add_argument("--dry-run", action="store_true", help="exercise the launcher and the rank plumbing on CPU (gloo), no kernels")
     args = ap.parse_args()
+
+    # no launcher around us: start the ranks ourselves
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        if not args.dry_run and args.impl == "ours":
+            import torch
+            have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+            if have < args.gpus:
+                raise SystemExit(f"bench.py --gpus {args.gpus} needs {args.gpus} CUDA devices, this host has {have}")
+        raise SystemExit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.dry_run:
+        run_dry(args)
+        return
 
     from paper_2605_02888_b200 import synth
     w = synth.WORKLOADS[args.workload]
@@ -200,9 +275,13 @@ def main():
         from paper_2605_02888_b200 import binding
         binding._lib = binding.load_library(args.lib)
 
+    from paper_2605_02888_b200 import binding as _b
+    flags = (_b.READ_ALL_TARGET_ROWS if args.no_early_exit else 0) | \
+            {"auto": 0, "stream": _b.SCHEDULE_STREAM, "sliced": _b.SCHEDULE_SLICED}[args.schedule]
+
     def gpu_batch(s):
         return speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],
-                            gamma=s["gamma"], temperature=s["temperature"], uniforms=s["uniforms"])
+                            gamma=s["gamma"], temperature=s["temperature"], uniforms=s["uniforms"], flags=flags)
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
@@ -237,24 +316,38 @@ def main():
     torch.cuda.synchronize()
     if dist:
         dist.barrier()
+    # The timed region: blocks of exactly `steps` steps, each bracketed by CUDA events, repeated until
+    # min_seconds have passed (so that the region is long enough for the clock record whatever `steps`
+    # is); every block's time is the MAX over the ranks; the reported block is the median one.
     sampler = ClockSampler(local)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
-    e0.record()
-    for i in range(args.steps):
-        one(i)
-    e1.record()
-    torch.cuda.synchronize()
+    blocks_ms = []
+    t_wall = time.perf_counter()
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            one(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1)
+        more = 1.0 if (time.perf_counter() - t_wall < args.min_seconds and len(blocks_ms) < 9999) else 0.0
+        if dist:
+            t = torch.tensor([ms, more], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms, more = float(t[0].item()), float(t[1].item())
+        blocks_ms.append(ms)
+        if not more:
+            break
     clocks = sampler.stop()
-    ms_total = e0.elapsed_time(e1)
     if dist:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
         dist.barrier()
+    ms_total = statistics.median(blocks_ms)
     ms_step = ms_total / args.steps
     value = w.B * world / (ms_step * 1e-3)
+    if clocks.get("sm_mhz"):
+        clocks["ms_per_step_x_sm_mhz"] = ms_step * clocks["sm_mhz"]
 
     # dominant kernel alone: events recorded by the library around the sweep kernel
     n_prof = min(args.steps, 200)
@@ -271,8 +364,11 @@ def main():
     # the library picks by logit type and batch: fp32, 384..1024 rows -> ring sweep, then a resample kernel (two launches per step);
     # bf16 -> register-staged sweep whose grid also carries the resample CTAs (one launch per step, so
     # its duration is that of the whole pass over the batch, second read of the stop positions included)
-    kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024) else "sweep_kernel"
-    one_launch = kernel == "sweep_kernel"
+    if args.schedule == "stream":
+        kernel = "stream_kernel"
+    else:
+        kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024) else "sweep_kernel"
+    one_launch = kernel != "pipe_sweep_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,
                 "algorithmic_bytes_per_launch": bytes_avg, "kernel_ms": sweep_avg,
@@ -328,10 +424,27 @@ def main():
         del host, devbuf
 
     cpu_baseline = None
+    parity = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import numpy as np
         import oracle
-        from parity import oracle_batch
+        from parity import compare_step, oracle_batch
         cores = host_cores()
+        # evidence that the timed outputs are the right ones: the last step of each resident batch, as the
+        # timed loop left it, against the oracle on a fixed sample of rows (mismatches outside the oracle's
+        # near-tie flags raise; the counts go into the line)
+        prow = np.unique(np.linspace(0, w.B - 1, num=min(w.B, 32)).astype(np.int64))
+        mwc = synth.make_mlp(wr, "cpu")
+        omc = oracle.Mlp(*(mwc[k2].numpy() for k2 in ("W1", "b1", "W2", "b2")))
+        parity = {"rows": 0, "n_accepted_mismatch": 0, "token_mismatch": 0, "gamma_mismatch": 0, "near_accept_rows": 0,
+                  "near_cdf_rows": 0, "near_cdf_abs_rows": 0, "near_gamma_rows": 0, "small_residual_rows": 0}
+        for k in range(n_batches):
+            compk = steps_in[k]["comp"].cpu().numpy()[prow]
+            ref = oracle.step(oracle_batch(steps_in[k], rows=prow, n_threads=cores), compk, omc)
+            rep = compare_step(outs[k].as_dict(), ref, rows=prow, mlp=omc, comp=compk)
+            for kk in parity:
+                parity[kk] += rep.get(kk, 0)
+        parity["against"] = "oracle, %d sampled rows of each resident batch after the timed loop" % len(prow)
         # bounded sample: whole batches of the resident steps, repeated until about 12 s of CPU work
         # are done (rows per batch capped so that one call stays near a second)
         rows = list(range(min(w.B, 256)))
@@ -353,14 +466,12 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "B_per_gpu": w.B, "gamma_max": w.gamma_max, "V": w.V,
-                       "logits": w.dtype, "temperature": w.temperature,
-                       "gamma_per_row": {"choices": "hash-uniform over {2,4,6,8}", "ragged": "hash-uniform over 1..gamma_max"}.get(
-                           w.gamma_mode, f"{min(w.gamma_fixed, w.gamma_max)} for every row"),
-                       "temperature_mode": w.temperature_mode, "mean_gamma": float(gam.float().mean()),
-                       "l2": f"{n_batches} resident batches of {bytes_step[0] / 1e6:.0f} MB alternate (each larger than L2)",
-                       "parallelism": f"dp{world} (rows sharded, no collective)"},
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
+            "config": dict(config_of(w), mean_gamma=float(gam.float().mean()),
+                           l2=f"{n_batches} resident batches of {bytes_step[0] / 1e6:.0f} MB alternate (each larger than L2)",
+                           parallelism=f"dp{world} (rows sharded, no collective)",
+                           early_exit=not args.no_early_exit, schedule=args.schedule),
+            "timed_blocks": len(blocks_ms), "ms_per_block_median": ms_total,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "parity": parity, "e2e": e2e, "clocks": clocks,
             "gpu_launches": (1 if one_launch else 2) * args.steps,
             "tokens_per_step_mean": float(outs[0].n_accepted.float().mean()) + 1.0,
         }))

@@ -37,6 +37,15 @@ int speckv_internal_set_wait_limit(int polls);
 speckv_status speckv_internal_wait_probe(int32_t B, int32_t* row_status, int32_t* out_tokens, void* workspace,
                                          size_t workspace_bytes, void* cuda_stream);
 
+/* Bounds-checked build only (the library built with -DSPECKV_DEBUG, `python -m paper_2605_02888_b200.build
+ * --debug`; the ordinary build returns SPECKV_ERR_UNSUPPORTED).  In that build every kernel compares the
+ * address of each logit load and of each workspace access with the extents of the call's buffers, and
+ * skips and counts an access that lies outside.  This call synchronises the device and returns
+ * out4 = {violations so far, address of the first one, its size in bytes, its kind}; reset != 0 clears
+ * the record afterwards; selftest != 0 first has a kernel check two addresses that no call registered
+ * (they are only compared, never dereferenced), so that the record must then show violations.        */
+speckv_status speckv_internal_debug_report(unsigned long long* out4, int reset, int selftest);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,7 @@ _LIB = os.path.join(_HERE, "libspeckv_oracle.so")
 
 DT_F32, DT_BF16 = 0, 1
 ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE = 0, 1, 2, 4, 8
-NEAR_ACCEPT, NEAR_CDF, NEAR_GREEDY, NEAR_GAMMA, NEAR_SMALL_RESIDUAL = 1, 2, 4, 8, 16
+NEAR_ACCEPT, NEAR_CDF, NEAR_GREEDY, NEAR_GAMMA, NEAR_SMALL_RESIDUAL, NEAR_CDF_ABS = 1, 2, 4, 8, 16, 32
 
 
 def build(force: bool = False) -> str:

@@ -140,13 +140,18 @@ int32_t inverse_cdf(const double* w, int32_t V, double u, int32_t* near_boundary
         return chosen;
     }
     if (near_boundary) {
-        const double eps = 1e-6 * W;
         /* upper boundary of the chosen token, and its lower boundary (= upper boundary of
          * the previous token with positive weight); the lower one only matters if a token
-         * with positive weight precedes the chosen one */
-        bool near_hi = std::fabs(cum - tau) < eps;
-        bool near_lo = (lower > 0.0) && std::fabs(tau - lower) < eps;
-        *near_boundary = (near_hi || near_lo) ? 1 : 0;
+         * with positive weight precedes the chosen one.
+         * bit 0: a boundary within 1e-6 of the threshold on the normalised CDF (1e-6 * W);
+         * bit 1: within 1e-6 in the units of the weights themselves.  For weights that are probabilities
+         * (W = 1) the two coincide; for a residual max(0, p - q) of small mass W the second is the wider
+         * one: p and q are each known to about 1e-7 when the sums behind them are accumulated in fp32,
+         * so their difference is known to about 1e-7 however small W is. */
+        const double d_hi = std::fabs(cum - tau);
+        const double d_lo = (lower > 0.0) ? std::fabs(tau - lower) : 1e300;
+        const double d = std::min(d_hi, d_lo);
+        *near_boundary = (d < 1e-6 * W ? 1 : 0) | (d < 1e-6 ? 2 : 0);
     }
     return chosen;
 }
@@ -432,7 +437,8 @@ void verify_row(const oracle_batch* bt, int32_t b, int32_t* n_accepted, int32_t*
         } else {
             fresh = inverse_cdf(p.data(), V, u2, &nb);
         }
-        if (nb) nearbits |= ORACLE_NEAR_CDF;
+        if (nb & 1) nearbits |= ORACLE_NEAR_CDF;
+        else if (nb & 2) nearbits |= ORACLE_NEAR_CDF_ABS;
     }
 
     n_accepted[b] = n;
@@ -475,7 +481,9 @@ int oracle_softmax_row(const void* row, int32_t dtype, int32_t V, double T, doub
 double oracle_entropy_nats(const double* prob, int32_t V) { return entropy_nats(prob, V); }
 
 int32_t oracle_inverse_cdf(const double* w, int32_t V, double u, int32_t* near_boundary) {
-    return inverse_cdf(w, V, u, near_boundary);
+    const int32_t tok = inverse_cdf(w, V, u, near_boundary);
+    if (near_boundary) *near_boundary &= 1;
+    return tok;
 }
 
 int32_t oracle_argmax_row(const void* row, int32_t dtype, int32_t V) {
@@ -539,7 +547,7 @@ int oracle_sample_draft(const oracle_batch* bt, const float* uniforms, int32_t* 
                 if (!softmax_row(draft_row(bt, b, i), V, rp.T, q.data())) { status |= ORACLE_ROW_NONFINITE; break; }
                 int32_t nb = 0;
                 tok[i] = inverse_cdf(q.data(), V, static_cast<double>(uniforms[static_cast<int64_t>(b) * G + i]), &nb);
-                if (nb) nearbits |= ORACLE_NEAR_CDF;
+                if (nb & 1) nearbits |= ORACLE_NEAR_CDF;
             }
         }
         if (!status) std::copy(tok.begin(), tok.end(), tb);

@@ -41,6 +41,8 @@ extern "C" {
 #define ORACLE_NEAR_GREEDY 4 /* (unused for exact ties: those resolve by lowest index)   */
 #define ORACLE_NEAR_GAMMA 8  /* best and second-best controller score within 1e-5 rel.   */
 #define ORACLE_NEAR_SMALL_RESIDUAL 16 /* rejected position whose residual mass is below 1e-5 */
+#define ORACLE_NEAR_CDF_ABS 32        /* residual draw: threshold within 1e-6 of a boundary in units of probability
+                                         (not of the residual's own mass W, which bit 2 measures)            */
 
 typedef struct {
     int32_t B;         /* rows (sequences) in the batch                                  */

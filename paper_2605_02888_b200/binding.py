@@ -92,6 +92,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     L.speckv_internal_set_wait_limit.argtypes = [C.c_int]
     L.speckv_internal_wait_probe.restype = C.c_int
     L.speckv_internal_wait_probe.argtypes = [C.c_int32, vp, vp, vp, sz, vp]
+    L.speckv_internal_debug_report.restype = C.c_int
+    L.speckv_internal_debug_report.argtypes = [C.POINTER(C.c_ulonglong), C.c_int, C.c_int]
     i32, i64 = C.c_int32, C.c_int64
     L.speckv_shard_workspace_size.restype = C.c_int
     L.speckv_shard_workspace_size.argtypes = [C.POINTER(_CBatch), C.POINTER(sz)]
@@ -132,6 +134,23 @@ def _dev_ptr(t: Optional[torch.Tensor], dtype: torch.dtype, name: str):
     return t.data_ptr()
 
 
+def _buf(t: Optional[torch.Tensor], dtype: torch.dtype, shape: tuple, dev: torch.device, name: str):
+    """Pointer of a caller-provided buffer after checking what the library cannot: exact shape, dtype,
+    contiguity and that it lives on the logits' device (a wrong one would be an out-of-bounds or
+    foreign-address write on the GPU).  None passes through as NULL."""
+    if t is None:
+        return None
+    if not t.is_cuda or t.device != dev:
+        raise ValueError(f"{name} must be on {dev}, got {t.device}")
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name} must have shape {tuple(shape)}, got {tuple(t.shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
 @dataclass
 class Batch:
     """One speculation step's inputs as CUDA tensors (see speckv_batch in speckv.h)."""
@@ -167,7 +186,7 @@ class Batch:
         c.draft_stride_b, c.draft_stride_pos = d.stride(0), d.stride(1)
         t = self.target_logits
         if t is not None:
-            if tuple(t.shape) != (B, G + 1, V) or t.dtype != d.dtype or not t.is_cuda:
+            if tuple(t.shape) != (B, G + 1, V) or t.dtype != d.dtype or not t.is_cuda or t.device != d.device:
                 raise ValueError("target_logits must be a CUDA tensor [B, gamma_max+1, V] of the draft's dtype")
             if V > 1 and t.stride(2) != 1:
                 raise ValueError("the vocabulary dimension must be contiguous")
@@ -176,9 +195,7 @@ class Batch:
         for name, dt, shp in (("draft_tokens", torch.int32, (B, G)), ("gamma", torch.int32, (B,)),
                               ("temperature", torch.float32, (B,)), ("uniforms", torch.float32, (B, G + 1, 2))):
             a = getattr(self, name)
-            if a is not None and tuple(a.shape) != shp:
-                raise ValueError(f"{name} must have shape {shp}, got {tuple(a.shape)}")
-            setattr(c, name, _dev_ptr(a, dt, name))
+            setattr(c, name, _buf(a, dt, shp, d.device, name))
         c.temperature_scalar = float(self.temperature_scalar)
         c.entropy_in_bits = int(bool(self.entropy_in_bits))
         c.flags = int(self.flags)
@@ -282,15 +299,36 @@ class StepOutputs:
         return {k: getattr(self, k) for k in ("H", "C", "feat", "scores", "gamma_next", "n_accepted",
                                               "out_tokens", "row_status")}
 
+    def pointers(self, batch: "Batch", n_out: int) -> dict:
+        """Device pointers of the buffers, each checked against the batch it is about to be used with."""
+        B, G, V = batch.shape()
+        dev = batch.draft_logits.device
+        f32, i32 = torch.float32, torch.int32
+        p = dict(H=_buf(self.H, f32, (B, G), dev, "H"), C=_buf(self.C, f32, (B, G), dev, "C"),
+                 feat=_buf(self.feat, f32, (B, 4), dev, "feat"),
+                 scores=_buf(self.scores, f32, (B, n_out), dev, "scores") if n_out else None,
+                 gamma_next=_buf(self.gamma_next, i32, (B,), dev, "gamma_next"),
+                 n_accepted=_buf(self.n_accepted, i32, (B,), dev, "n_accepted"),
+                 out_tokens=_buf(self.out_tokens, i32, (B, G + 1), dev, "out_tokens"),
+                 row_status=_buf(self.row_status, i32, (B,), dev, "row_status"))
+        ws = self.workspace
+        if ws is None or not ws.is_cuda or ws.device != dev or ws.dtype != torch.uint8 or not ws.is_contiguous():
+            raise ValueError(f"workspace must be a contiguous uint8 tensor on {dev}")
+        if ws.numel() < workspace_size(batch):
+            raise ValueError(f"workspace holds {ws.numel()} bytes, this batch needs {workspace_size(batch)}")
+        p["workspace"] = ws.data_ptr()
+        return p
+
 
 def speckv_signals(batch: Batch, out: Optional[StepOutputs] = None):
     """Draft signals (paper Sec. 4.2): H, C [B, gamma_max]; feat [B, 4]; row_status [B]."""
     L = load_library()
     c = batch._c()
     o = out or StepOutputs.allocate(batch)
+    q = o.pointers(batch, 0)
     with torch.cuda.device(batch.draft_logits.device):
-        rc = L.speckv_signals(C.byref(c), _ptr(o.H), _ptr(o.C), _ptr(o.feat), _ptr(o.row_status),
-                              _ptr(o.workspace), o.workspace.numel(), _stream(batch.draft_logits.device))
+        rc = L.speckv_signals(C.byref(c), q["H"], q["C"], q["feat"], q["row_status"],
+                              q["workspace"], o.workspace.numel(), _stream(batch.draft_logits.device))
     if rc != OK:
         raise SpeckvError(rc, "speckv_signals")
     return dict(H=o.H, C=o.C, feat=o.feat, row_status=o.row_status)
@@ -305,10 +343,12 @@ def speckv_signals_static(batch: Batch, H: torch.Tensor, Cc: torch.Tensor, feat:
     L = load_library()
     c = batch._c()
     dev = batch.draft_logits.device
+    B, G, _ = batch.shape()
+    f32 = torch.float32
+    ptrs = (_buf(H, f32, (B, G), dev, "H"), _buf(Cc, f32, (B, G), dev, "C"), _buf(feat, f32, (B, 4), dev, "feat"),
+            _buf(row_status, torch.int32, (B,), dev, "row_status"))
     with torch.cuda.device(dev):
-        rc = L.speckv_signals_static(C.byref(c), _dev_ptr(H, torch.float32, "H"), _dev_ptr(Cc, torch.float32, "C"),
-                                     _dev_ptr(feat, torch.float32, "feat"),
-                                     _dev_ptr(row_status, torch.int32, "row_status"), _stream(dev))
+        rc = L.speckv_signals_static(C.byref(c), *ptrs, _stream(dev))
     if rc != OK:
         raise SpeckvError(rc, "speckv_signals_static")
     return dict(H=H, C=Cc, feat=feat, row_status=row_status)
@@ -322,8 +362,7 @@ def speckv_sample_draft(batch: Batch, uniforms: torch.Tensor, tokens: Optional[t
     c = batch._c()
     B, G, V = batch.shape()
     dev = batch.draft_logits.device
-    if tuple(uniforms.shape) != (B, G):
-        raise ValueError(f"uniforms must have shape {(B, G)}")
+    _buf(uniforms, torch.float32, (B, G), dev, "uniforms")
     if tokens is None:
         tokens = torch.empty(B, G, dtype=torch.int32, device=dev)
     if row_status is None:
@@ -335,9 +374,10 @@ def speckv_sample_draft(batch: Batch, uniforms: torch.Tensor, tokens: Optional[t
             raise SpeckvError(rc, "speckv_sample_workspace_size")
         workspace = torch.empty(int(n.value), dtype=torch.uint8, device=dev)
     with torch.cuda.device(dev):
-        rc = L.speckv_sample_draft(C.byref(c), _dev_ptr(uniforms, torch.float32, "uniforms"),
-                                   _dev_ptr(tokens, torch.int32, "tokens"), _dev_ptr(row_status, torch.int32, "row_status"),
-                                   _ptr(workspace), workspace.numel(), _stream(dev))
+        rc = L.speckv_sample_draft(C.byref(c), _buf(uniforms, torch.float32, (B, G), dev, "uniforms"),
+                                   _buf(tokens, torch.int32, (B, G), dev, "tokens"),
+                                   _buf(row_status, torch.int32, (B,), dev, "row_status"),
+                                   _buf(workspace, torch.uint8, (workspace.numel(),), dev, "workspace"), workspace.numel(), _stream(dev))
     if rc != OK:
         raise SpeckvError(rc, "speckv_sample_draft")
     return dict(tokens=tokens, row_status=row_status)
@@ -354,9 +394,13 @@ def speckv_select_gamma(feat: torch.Tensor, comp: Optional[torch.Tensor], mlp: M
         scores = torch.empty(B, mlp.n_out, dtype=torch.float32, device=dev)
     if gamma_next is None:
         gamma_next = torch.empty(B, dtype=torch.int32, device=dev)
+    if not feat.is_cuda:
+        raise ValueError("feat must be a CUDA tensor (the library has no CPU path)")
     with torch.cuda.device(dev):
-        rc = L.speckv_select_gamma(B, _dev_ptr(feat, torch.float32, "feat"), _dev_ptr(comp, torch.float32, "comp"),
-                                   C.byref(m), _ptr(scores), _ptr(gamma_next), _stream(dev))
+        rc = L.speckv_select_gamma(B, _buf(feat, torch.float32, (B, 4), dev, "feat"),
+                                   _buf(comp, torch.float32, (B, mlp.n_comp), dev, "comp") if mlp.n_comp > 0 else None,
+                                   C.byref(m), _buf(scores, torch.float32, (B, mlp.n_out), dev, "scores"),
+                                   _buf(gamma_next, torch.int32, (B,), dev, "gamma_next"), _stream(dev))
     if rc != OK:
         raise SpeckvError(rc, "speckv_select_gamma")
     return dict(scores=scores, gamma_next=gamma_next)
@@ -368,9 +412,10 @@ def speckv_verify(batch: Batch, out: Optional[StepOutputs] = None):
     c = batch._c()
     o = out or StepOutputs.allocate(batch)
     dev = batch.draft_logits.device
+    q = o.pointers(batch, 0)
     with torch.cuda.device(dev):
-        rc = L.speckv_verify(C.byref(c), _ptr(o.n_accepted), _ptr(o.out_tokens), _ptr(o.row_status),
-                             _ptr(o.workspace), o.workspace.numel(), _stream(dev))
+        rc = L.speckv_verify(C.byref(c), q["n_accepted"], q["out_tokens"], q["row_status"],
+                             q["workspace"], o.workspace.numel(), _stream(dev))
     if rc != OK:
         raise SpeckvError(rc, "speckv_verify")
     return dict(n_accepted=o.n_accepted, out_tokens=o.out_tokens, row_status=o.row_status)
@@ -387,9 +432,14 @@ def speckv_step(batch: Batch, comp: Optional[torch.Tensor], mlp: Mlp, out: Optio
     m = mlp._c()
     o = out or StepOutputs.allocate(batch, mlp.n_out)
     dev = batch.draft_logits.device
-    args = [C.byref(c), _dev_ptr(comp, torch.float32, "comp"), C.byref(m), _ptr(o.H), _ptr(o.C),
-            _ptr(o.feat), _ptr(o.scores), _ptr(o.gamma_next), _ptr(o.n_accepted),
-            _ptr(o.out_tokens), _ptr(o.row_status), _ptr(o.workspace), o.workspace.numel(), _stream(dev)]
+    q = o.pointers(batch, mlp.n_out)
+    B = batch.shape()[0]
+    cptr = _buf(comp, torch.float32, (B, mlp.n_comp), dev, "comp") if (comp is not None and mlp.n_comp > 0) else None
+    for name in ("W1", "b1", "W2", "b2"):
+        if getattr(mlp, name).device != dev:
+            raise ValueError(f"controller parameter {name} must be on {dev}")
+    args = [C.byref(c), cptr, C.byref(m), q["H"], q["C"], q["feat"], q["scores"], q["gamma_next"], q["n_accepted"],
+            q["out_tokens"], q["row_status"], q["workspace"], o.workspace.numel(), _stream(dev)]
     with torch.cuda.device(dev):
         if events is None:
             rc = L.speckv_step(*args)

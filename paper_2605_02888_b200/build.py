@@ -24,28 +24,34 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+DEBUG_LIB_PATH = os.path.join(_CSRC, "libspeckv_debug.so")
+
+
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     deps = [os.path.join(_CSRC, d) for d in _DEPS] + [os.path.join(_INC, h) for h in ("speckv.h", "speckv_internal.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the library if it is missing or older than its sources; return its path."""
-    if not force and not is_stale():
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", _INC, "-o", tmp] + [os.path.join(_CSRC, s) for s in _SOURCES]
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile the library if it is missing or older than its sources; return its path.
+    debug=True builds the bounds-checked variant (-DSPECKV_DEBUG) beside it: every logit load and
+    workspace access is compared with the call's extents, skipped and counted when outside."""
+    out = DEBUG_LIB_PATH if debug else LIB_PATH
+    if not force and not is_stale(out):
+        return out
+    tmp = out + f".tmp{os.getpid()}"
+    cmd = [_nvcc(), *NVCC_FLAGS, *(["-DSPECKV_DEBUG"] if debug else []), "-I", _INC, "-o", tmp] + [os.path.join(_CSRC, s) for s in _SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")
         print(" ".join(cmd), file=sys.stderr)
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out)
+    return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

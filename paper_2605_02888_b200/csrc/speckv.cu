@@ -22,9 +22,7 @@ namespace {
 
 using namespace speckv;
 
-#ifndef SPECKV_SLICE_BYTES
-#define SPECKV_SLICE_BYTES 262144 // bytes of one logit row that one sweep CTA streams
-#endif
+constexpr int kSliceBytes = 262144;  // bytes of one logit row that one sweep CTA streams
 constexpr size_t kAlign = 256;
 // upper bound of a verification step's logit bytes from which the stream kernel is taken
 constexpr long long kStreamMinBytes = 128ll << 20;
@@ -42,11 +40,43 @@ struct Plan {
 
 inline int esize(speckv_dtype dt) { return dt == SPECKV_BF16 ? 2 : 4; }
 
+// Bounds-checked build: the extents a call's kernels may touch, registered on the call's stream before
+// its first kernel.  Range 0: draft logits, 1: target logits, 2: workspace, 3..: further caller arrays.
+struct DbgExtra { const void* p; size_t bytes; };
+cudaError_t dbg_register(cudaStream_t cs, const speckv_batch* bt, bool target, const void* ws, size_t ws_bytes,
+                         const DbgExtra* extra = nullptr, int n_extra = 0) {
+#ifdef SPECKV_DEBUG
+    DbgRanges r{};
+    auto span = [&](const void* base, int64_t sb, int64_t sp, int n_pos) -> unsigned long long {
+        const long long last = static_cast<long long>(bt->B - 1) * sb + static_cast<long long>(n_pos - 1) * sp + bt->V;
+        return reinterpret_cast<unsigned long long>(base) + static_cast<unsigned long long>(last) * esize(bt->dtype);
+    };
+    if (bt->B > 0 && bt->draft_logits) {
+        r.lo[0] = reinterpret_cast<unsigned long long>(bt->draft_logits);
+        r.hi[0] = span(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, bt->gamma_max);
+    }
+    if (bt->B > 0 && target && bt->target_logits) {
+        r.lo[1] = reinterpret_cast<unsigned long long>(bt->target_logits);
+        r.hi[1] = span(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, bt->gamma_max + 1);
+    }
+    r.lo[2] = reinterpret_cast<unsigned long long>(ws);
+    r.hi[2] = r.lo[2] + ws_bytes;
+    for (int k = 0; k < n_extra && 3 + k < kDbgRanges; ++k) {
+        r.lo[3 + k] = reinterpret_cast<unsigned long long>(extra[k].p);
+        r.hi[3 + k] = r.lo[3 + k] + extra[k].bytes;
+    }
+    return cudaMemcpyToSymbolAsync(g_dbg_ranges, &r, sizeof r, 0, cudaMemcpyHostToDevice, cs);
+#else
+    (void)cs; (void)bt; (void)target; (void)ws; (void)ws_bytes; (void)extra; (void)n_extra;
+    return cudaSuccess;
+#endif
+}
+
 // vocabulary slices per logit row for a sweep over J logit rows per batch row
 int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
     const int nvec = (V + kVec - 1) / kVec;
     const double row_bytes = static_cast<double>(V) * esize(dt);
-    int ns = static_cast<int>(std::lround(row_bytes / static_cast<double>(SPECKV_SLICE_BYTES)));
+    int ns = static_cast<int>(std::lround(row_bytes / static_cast<double>(kSliceBytes)));
     if (ns < 1) ns = 1;
     // small batches: enough CTAs to put a few on every SM
     const long long rows = static_cast<long long>(B) * J;
@@ -60,9 +90,7 @@ int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
     return ns;
 }
 
-#ifndef SPECKV_RS_CHUNKS
-#define SPECKV_RS_CHUNKS 64  // 256-element chunks of the stop position that one resample CTA sums
-#endif
+constexpr int kRsChunksPerCta = 64;  // 256-element chunks of the stop position that one resample CTA sums
 
 Plan make_plan(const speckv_batch* bt) {
     Plan p;
@@ -70,7 +98,7 @@ Plan make_plan(const speckv_batch* bt) {
     p.J_full = 2 * bt->gamma_max + 1;
     p.nvec = (bt->V + kVec - 1) / kVec;
     p.nchunk = (bt->V + kChunk - 1) / kChunk;
-    p.R = (p.nchunk + SPECKV_RS_CHUNKS - 1) / SPECKV_RS_CHUNKS;
+    p.R = (p.nchunk + kRsChunksPerCta - 1) / kRsChunksPerCta;
     if (p.R > 32) p.R = 32;
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
@@ -223,36 +251,25 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
     int sms = 0;
     e = sm_count(&sms);
     if (e != cudaSuccess) return e;
-    pipe_sweep_kernel<T><<<SPECKV_PIPE_CTAS * sms, kPipeThreads, smem, st>>>(P);
+    pipe_sweep_kernel<T><<<kPipeCtasPerSm * sms, kPipeThreads, smem, st>>>(P);
     return cudaGetLastError();
 }
 
-// 1: after the register-staged sweep the fresh tokens are drawn by extra CTAs of the same launch;
-// 0: always by a second kernel (measurement builds)
-// the rows swept last have their fresh tokens drawn by more, shorter CTAs (see resample_body)
-#ifndef SPECKV_RS_TAIL_ROWS
-#define SPECKV_RS_TAIL_ROWS 16
-#endif
-#ifndef SPECKV_RS_TAIL_MULT
-#define SPECKV_RS_TAIL_MULT 2
-#endif
-#ifndef SPECKV_RS_SMALL_CTAS
-#define SPECKV_RS_SMALL_CTAS 1184  // resample CTAs wanted in flight for a small batch (two per CTA slot)
-#endif
-#ifndef SPECKV_MERGED
-#define SPECKV_MERGED 1
-#endif
+// After the register-staged sweep the fresh tokens are drawn by extra CTAs of the same launch; the rows swept last have their fresh tokens drawn by more, shorter CTAs (see resample_body)
+constexpr int kRsTailRows = 16;
+constexpr int kRsTailMult = 2;
+constexpr int kRsSmallCtas = 1184;  // resample CTAs wanted in flight for a small batch (two per CTA slot)
 
 template <typename T, bool ALIGNED>
 cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged) {
-    constexpr int U = sizeof(T) == 2 ? SPECKV_U : (SPECKV_U + 1) / 2;
+    constexpr int U = sizeof(T) == 2 ? kSweepLoads : (kSweepLoads + 1) / 2;
     const bool verify = (P.mode & MODE_VERIFY) != 0;
     const bool ring = ALIGNED && staged;
     P.rs_tail = 0; P.R2 = P.R; P.chunks_per_cta2 = P.chunks_per_cta;
-    bool merged = SPECKV_MERGED && verify && !ring && P.rdone;
-    if (merged && P.B >= 4 * SPECKV_RS_TAIL_ROWS && P.R * SPECKV_RS_TAIL_MULT <= 32 && SPECKV_RS_TAIL_MULT > 1) {
-        P.rs_tail = SPECKV_RS_TAIL_ROWS;
-        P.R2 = P.R * SPECKV_RS_TAIL_MULT;
+    bool merged = verify && !ring && P.rdone;
+    if (merged && P.B >= 4 * kRsTailRows && P.R * kRsTailMult <= 32 && kRsTailMult > 1) {
+        P.rs_tail = kRsTailRows;
+        P.R2 = P.R * kRsTailMult;
         P.chunks_per_cta2 = (P.nchunk + P.R2 - 1) / P.R2;
     }
     const long long n_draw = static_cast<long long>(P.B - P.rs_tail) * P.R + static_cast<long long>(P.rs_tail) * P.R2;
@@ -340,7 +357,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     {
         // small batches: more, shorter shares per row, so that the draw of a handful of rows still spreads
         // over the SMs (the draw of a row is a chain of dependent round trips, shorter with fewer chunks per CTA)
-        const int want = (SPECKV_RS_SMALL_CTAS + P.B - 1) / P.B;
+        const int want = (kRsSmallCtas + P.B - 1) / P.B;
         int cap = (P.nchunk + 7) / 8;  // at least one chunk per warp
         if (cap > 32) cap = 32;
         if (want > P.R && cap > P.R) {
@@ -372,6 +389,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (dbg_register(cs, bt, verify, ws, ws_bytes) != cudaSuccess) return SPECKV_ERR_CUDA;
     const int es = esize(bt->dtype);
     bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
     if (verify) aligned = aligned && rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
@@ -417,17 +435,11 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     // exponential per two bytes, and hiding that latency next to the memory latency takes the 32
     // warps per SM of the register-staged kernel (4.95 against 4.6 TB/s), whose draining tail the
     // resample CTAs of the same grid then fill.
-#ifndef SPECKV_STAGED
-#define SPECKV_STAGED 1  // 0: never, 1: fp32 only, 2: whenever the layout allows (measurement builds)
-#endif
     // Below a few hundred rows the ring's fixed costs (per-CTA tables, one epilogue warp per CTA, a
     // resample kernel that cannot overlap) outweigh its streaming rate: b512_mixed cut to 128 / 256 /
     // 512 rows takes 178 / 317 / 564 us with the ring and 166 / 307 / 581 us without.
-#ifndef SPECKV_PIPE_MINB
-#define SPECKV_PIPE_MINB 384
-#endif
-    const bool staged = (SPECKV_STAGED == 2 || (SPECKV_STAGED == 1 && bt->dtype == SPECKV_F32)) && aligned &&
-                        row_bytes % 16 == 0 && P.B <= kPipeMaxB && (SPECKV_STAGED == 2 || P.B >= SPECKV_PIPE_MINB);
+constexpr int kPipeMinB = 384;
+    const bool staged = bt->dtype == SPECKV_F32 && aligned && row_bytes % 16 == 0 && P.B <= kPipeMaxB && P.B >= kPipeMinB;
     // completion flags per batch row and the logits at the draft tokens: only the register-staged sweep
     // overlaps the resample work with its own tail; after the ring sweep the resample kernel starts when
     // everything is done and a flag would only cost it a round trip
@@ -504,25 +516,21 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     P.n_sweep = P.B * P.J * P.nsplit;
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (dbg_register(cs, bt, false, ws, ws_bytes) != cudaSuccess) return SPECKV_ERR_CUDA;
     const size_t n_tick = static_cast<size_t>(P.B) * (2 + static_cast<size_t>(P.G));
     if (cudaMemsetAsync(P.tick1, 0, n_tick * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
     const int es = esize(bt->dtype);
     const bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
-#ifndef SPECKV_SAMPLE_CTAS
-#define SPECKV_SAMPLE_CTAS 2368
-#endif
-#ifndef SPECKV_SAMPLE_ONEPASS
-#define SPECKV_SAMPLE_ONEPASS 1  // 0: always normaliser sweep + second pass (measurement builds)
-#endif
+constexpr int kSampleCtas = 2368;
     // One pass (speckv_sample.cuh) whenever a row's chunk records fit the searching CTA's shared memory.
-    if (SPECKV_SAMPLE_ONEPASS && P.nchunk <= kRsStage &&
+    if (P.nchunk <= kRsStage &&
         static_cast<long long>(P.B) * P.G * P.R <= 0x7fffffffLL) {
         P.csum2 = reinterpret_cast<float*>(w + pl.off_cz);
         // shares per logit row: enough CTAs to fill the SMs a few times over, no more (a CTA costs a few
         // microseconds before its first load returns)
         {
             const long long draws = static_cast<long long>(P.B) * P.G;
-            long long S = (SPECKV_SAMPLE_CTAS + draws - 1) / draws;
+            long long S = (kSampleCtas + draws - 1) / draws;
             if (S > P.R) S = P.R;
             if (S < 1) S = 1;
             P.R = static_cast<int>(S);
@@ -541,11 +549,11 @@ speckv_status run_sample(const speckv_batch* bt, const float* uniforms, int32_t*
     // one launch: the draws' CTAs sit behind the sweep CTAs of the same grid and wait for their batch
     // row's flag (as in the verification step); two launches when the grid would not fit
     const long long n_draw = static_cast<long long>(P.B) * P.G * P.R;
-    const bool merged = SPECKV_MERGED && P.n_sweep + n_draw <= 0x7fffffffLL;
+    const bool merged = P.n_sweep + n_draw <= 0x7fffffffLL;
     if (merged) P.rs_reverse = 0; else P.rdone = nullptr;
     const unsigned grid1 = static_cast<unsigned>(P.n_sweep + (merged ? n_draw : 0));
     const unsigned grid2 = static_cast<unsigned>(n_draw);
-    constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
+    constexpr int Ub = kSweepLoads, Uf = (kSweepLoads + 1) / 2;
     if (bt->dtype == SPECKV_BF16) {
         if (aligned) { sweep_kernel<__nv_bfloat16, true, Ub><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<__nv_bfloat16, true><<<grid2, kThreads, 0, cs>>>(P); }
         else { sweep_kernel<__nv_bfloat16, false, Ub><<<grid1, kThreads, 0, cs>>>(P); if (!merged) resample_kernel<__nv_bfloat16, false><<<grid2, kThreads, 0, cs>>>(P); }
@@ -587,7 +595,7 @@ ShardPlan make_shard_plan(const speckv_batch* bt) {
     const size_t B = static_cast<size_t>(bt->B), J = 2 * static_cast<size_t>(bt->gamma_max) + 1;
     p.nvec = (bt->V + kVec - 1) / kVec;
     p.nchunk = (bt->V + kChunk - 1) / kChunk;
-    p.R = (p.nchunk + SPECKV_RS_CHUNKS - 1) / SPECKV_RS_CHUNKS;
+    p.R = (p.nchunk + kRsChunksPerCta - 1) / kRsChunksPerCta;
     if (p.R > 32) p.R = 32;
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
@@ -600,9 +608,7 @@ ShardPlan make_shard_plan(const speckv_batch* bt) {
     return p;
 }
 
-#ifndef SPECKV_SHARD_WARP_ROW_BYTES
-#define SPECKV_SHARD_WARP_ROW_BYTES 65536  // slice rows up to this size are swept by one warp each
-#endif
+constexpr int kShardWarpRowBytes = 65536;  // slice rows up to this size are swept by one warp each
 
 // what every shard call needs from the local batch
 speckv_status shard_params(const speckv_batch* bt, void* ws, size_t ws_bytes, KParams& P, ShardPlan& pl) {
@@ -748,6 +754,33 @@ speckv_status speckv_step_profiled(const speckv_batch* batch, const float* comp,
                n_accepted, out_tokens, row_status, workspace, workspace_bytes, cuda_stream, ev);
 }
 
+#ifdef SPECKV_DEBUG
+namespace {
+__global__ void dbg_selftest_kernel() {
+    // addresses that no call has registered: looked at, never dereferenced
+    dbg_ok(reinterpret_cast<const void*>(0x10ull), 16, DBG_LOGIT16);
+    dbg_ok(reinterpret_cast<const void*>(0x20ull), 4, DBG_WS_STORE);
+}
+}  // namespace
+#endif
+
+speckv_status speckv_internal_debug_report(unsigned long long* out4, int reset, int selftest) {
+#ifdef SPECKV_DEBUG
+    if (!out4) return SPECKV_ERR_INVALID_ARG;
+    if (selftest) dbg_selftest_kernel<<<1, 1>>>();
+    if (cudaDeviceSynchronize() != cudaSuccess) return SPECKV_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(out4, g_dbg_report, sizeof(unsigned long long) * 4) != cudaSuccess) return SPECKV_ERR_CUDA;
+    if (reset) {
+        const unsigned long long zero[4] = {0, 0, 0, 0};
+        if (cudaMemcpyToSymbol(g_dbg_report, zero, sizeof zero) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
+    return SPECKV_OK;
+#else
+    (void)out4; (void)reset; (void)selftest;
+    return SPECKV_ERR_UNSUPPORTED;
+#endif
+}
+
 int speckv_internal_set_wait_limit(int polls) {
     if (polls < 1) polls = 1;
     return g_wait_limit.exchange(polls);
@@ -767,6 +800,10 @@ speckv_status speckv_internal_wait_probe(int32_t B, int32_t* row_status, int32_t
     P.rdone = static_cast<int*>(workspace);
     P.tick2 = P.rdone + B;
     cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    {
+        speckv_batch none{};
+        if (dbg_register(cs, &none, false, workspace, workspace_bytes) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
     if (cudaMemsetAsync(workspace, 0, 2 * static_cast<size_t>(B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
     wait_probe_fill<<<(B + 255) / 256, 256, 0, cs>>>(P);
     resample_kernel<float, true><<<static_cast<unsigned>(B), kThreads, 0, cs>>>(P);
@@ -799,19 +836,24 @@ speckv_status speckv_shard_sweep(const speckv_batch* local, int64_t v_begin, flo
     P.state = reinterpret_cast<float4*>(shard_state);
     P.tokl = reinterpret_cast<float2*>(shard_tokl);
     cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    {
+        const DbgExtra ex[2] = {{shard_state, static_cast<size_t>(P.B) * P.J * sizeof(float4)},
+                                {shard_tokl, static_cast<size_t>(P.B) * P.G * sizeof(float2)}};
+        if (dbg_register(cs, local, true, workspace, workspace_bytes, ex, 2) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
     if (cudaMemsetAsync(P.tick1, 0, (3 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
     if (cudaMemsetAsync(shard_tokl, 0, static_cast<size_t>(P.B) * P.G * sizeof(float2), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
     const unsigned grid = static_cast<unsigned>(P.n_sweep);
-    constexpr int Ub = SPECKV_U, Uf = (SPECKV_U + 1) / 2;
+    constexpr int Ub = kSweepLoads, Uf = (kSweepLoads + 1) / 2;
     const bool al = shard_aligned(local);
     // A slice row is short (V / n_shards columns).  One CTA per short row is mostly overhead and the
     // ring sweep pays per logit row as well (segment hand-over to its epilogue warp), so rows of up to
     // 64 KB are swept by one warp each, all of them resident at once; wider slices take the
     // CTA-per-slice sweep.
     const long long row_bytes = static_cast<long long>(P.V) * esize(local->dtype);
-    if (row_bytes <= SPECKV_SHARD_WARP_ROW_BYTES) {
+    if (row_bytes <= kShardWarpRowBytes) {
         const unsigned g2 = static_cast<unsigned>((static_cast<long long>(P.B) * P.J + kWarps - 1) / kWarps);
         if (local->dtype == SPECKV_BF16) {
             if (al) shard_rows_kernel<__nv_bfloat16, true, Ub><<<g2, kThreads, 0, cs>>>(P);
@@ -868,6 +910,13 @@ speckv_status speckv_shard_finish(const speckv_batch* local, int32_t n_shards, i
     P.info = static_cast<RowInfo*>(row_info);
     if (static_cast<long long>(P.B) * P.J > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
     const unsigned grid = static_cast<unsigned>((P.B + kWarps - 1) / kWarps);
+    {
+        speckv_batch none{};  // this call reads no logits: only the gathered arrays and the row records
+        const DbgExtra ex[3] = {{all_state, static_cast<size_t>(n_shards) * P.B * P.J * sizeof(float4)},
+                                {all_tokl, static_cast<size_t>(n_shards) * P.B * P.G * sizeof(float2)},
+                                {row_info, static_cast<size_t>(P.B) * sizeof(RowInfo)}};
+        if (dbg_register(static_cast<cudaStream_t>(cuda_stream), &none, false, nullptr, 0, ex, 3) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
     shard_finish_kernel<float><<<grid, kThreads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(P);
     return cudaGetLastError() == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
 }
@@ -882,6 +931,10 @@ speckv_status speckv_shard_draw_sums(const speckv_batch* local, const void* row_
     P.info = static_cast<RowInfo*>(const_cast<void*>(row_info));
     P.weight = shard_weight;
     cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    {
+        const DbgExtra ex[1] = {{row_info, static_cast<size_t>(P.B) * sizeof(RowInfo)}};
+        if (dbg_register(cs, local, true, workspace, workspace_bytes, ex, 1) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
     if (cudaMemsetAsync(P.tick2, 0, static_cast<size_t>(P.B) * sizeof(int), cs) != cudaSuccess) return SPECKV_ERR_CUDA;
     if (static_cast<long long>(P.B) * P.R > 0x7fffffffLL) return SPECKV_ERR_UNSUPPORTED;
     const unsigned grid = static_cast<unsigned>(P.B) * static_cast<unsigned>(P.R);
@@ -911,6 +964,10 @@ speckv_status speckv_shard_draw_pick(const speckv_batch* local, int64_t v_begin,
     P.out_tok = out_tokens;
     P.rank = rank; P.n_shards = n_shards; P.v_begin = static_cast<int>(v_begin);
     cudaStream_t cs = static_cast<cudaStream_t>(cuda_stream);
+    {
+        const DbgExtra ex[1] = {{row_info, static_cast<size_t>(P.B) * sizeof(RowInfo)}};
+        if (dbg_register(cs, local, true, workspace, workspace_bytes, ex, 1) != cudaSuccess) return SPECKV_ERR_CUDA;
+    }
     const unsigned grid = static_cast<unsigned>(P.B);
     const bool al = shard_aligned(local);
     if (local->dtype == SPECKV_BF16) {

@@ -27,16 +27,40 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kVec = 8;                 // elements per lane per step
 constexpr int kChunk = 32 * kVec;       // one warp step = one inverse-CDF chunk (256 elements)
 constexpr int kMaxSplit = 32;
-#ifndef SPECKV_U
-#define SPECKV_U 4            // 16-byte loads in flight per thread (bf16); fp32 uses half as many vector steps
-#endif
-#ifndef SPECKV_MINB
-#define SPECKV_MINB 4         // CTAs per SM the sweep kernel is compiled for
-#endif
+constexpr int kSweepLoads = 4;  // 16-byte loads in flight per thread (bf16); fp32 uses half as many vector steps
+constexpr int kSweepCtasPerSm = 4;  // CTAs per SM the sweep kernel is compiled for
 constexpr float kFloor = -1.2676506002282294e30f;  // -2^100: logits below count as -inf
 constexpr uint32_t kFloorBf16x2 = 0xF180F180u;     // -2^100 as two bf16
 constexpr double kLn2 = 0.6931471805599453094;
 constexpr double kLog2e = 1.4426950408889634074;
+
+// ---- bounds-checked build (-DSPECKV_DEBUG) ---------------------------------------------------------
+// Every global-memory access whose address comes out of index arithmetic (the logit loads of every
+// kernel, the reads and writes of the workspace, the reads of the caller's state arrays in the sharded
+// step) is first compared with the extents the host registered for the call.  An access outside them
+// is counted, its address kept, and NOT performed: loads give a neutral value, stores are dropped.
+// Nothing traps.  In the ordinary build the check is the constant true.
+constexpr int kDbgRanges = 8;
+struct DbgRanges { unsigned long long lo[kDbgRanges], hi[kDbgRanges]; };
+#ifdef SPECKV_DEBUG
+__device__ DbgRanges g_dbg_ranges;
+__device__ unsigned long long g_dbg_report[4];  // violations, first offending address, its size, the kind of access
+__device__ __forceinline__ bool dbg_ok(const void* p, unsigned bytes, int kind) {
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+#pragma unroll
+    for (int k = 0; k < kDbgRanges; ++k)
+        if (a >= g_dbg_ranges.lo[k] && a + bytes <= g_dbg_ranges.hi[k]) return true;
+    if (atomicAdd(&g_dbg_report[0], 1ull) == 0ull) {
+        g_dbg_report[1] = a;
+        g_dbg_report[2] = bytes;
+        g_dbg_report[3] = static_cast<unsigned long long>(kind);
+    }
+    return false;
+}
+#else
+__device__ __forceinline__ bool dbg_ok(const void*, unsigned, int) { return true; }
+#endif
+enum : int { DBG_LOGIT16 = 1, DBG_LOGIT1 = 2, DBG_WS_LOAD = 3, DBG_WS_STORE = 4, DBG_COPY = 5 };
 
 enum : int { MODE_SIGNALS = 1, MODE_VERIFY = 2, MODE_MLP = 4, MODE_SAMPLE = 8 };
 enum : int { PATH_DRAFT = 0, PATH_TARGET = 1, PATH_ARGMAX = 2 };
@@ -149,6 +173,7 @@ __device__ __forceinline__ float max_nan(float a, float b) {  // NaN-propagating
 }
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     uint4 v;
+    if (!dbg_ok(p, 16, DBG_LOGIT16)) return make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
@@ -204,9 +229,13 @@ __device__ __forceinline__ void unpack_pairs(const Raw<float>& r, f2 (&x)[4]) {
 }
 
 __device__ __forceinline__ float elem_to_float(const __nv_bfloat16* p, long long i) {
+    if (!dbg_ok(p + i, 2, DBG_LOGIT1)) return 0.f;
     return __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const unsigned short*>(p)[i]) << 16);
 }
-__device__ __forceinline__ float elem_to_float(const float* p, long long i) { return p[i]; }
+__device__ __forceinline__ float elem_to_float(const float* p, long long i) {
+    if (!dbg_ok(p + i, 4, DBG_LOGIT1)) return 0.f;
+    return p[i];
+}
 
 // kVec elements starting at element e0 of a row; elements at or beyond `hi` read as `pad`.
 // ALIGNED: the row is 16-byte aligned, so a full vector is one (bf16) or two (fp32) 16-byte loads.
@@ -605,7 +634,12 @@ __device__ __forceinline__ float4 sweep_warp(const T* __restrict__ row, int lo, 
 // ----------------------------------------------------------------------------------------
 // Row epilogue helpers (one warp, double precision; a few dozen values per row)
 // ----------------------------------------------------------------------------------------
-__device__ __forceinline__ float4 ldcg4(const float4* p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ldcg4(const float4* p) {
+    if (!dbg_ok(p, 16, DBG_WS_LOAD)) return make_float4(0.f, 0.f, 0.f, 0.f);
+    return __ldcg(p);
+}
+// a store into the workspace (or a caller's state array) at an index that was computed
+#define SPECKV_ST(lvalue, value) do { if (dbg_ok(&(lvalue), sizeof(lvalue), DBG_WS_STORE)) (lvalue) = (value); } while (0)
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -722,13 +756,10 @@ __device__ __forceinline__ void ctl_eval(const KParams& P, const CtlRegs& c, con
     if (gamma_next && lane == 0) *gamma_next = P.gch[best_j];
 }
 
-// log2 of a positive finite number as an exact integer part plus the fp32 log2 of the mantissa
-// (below one in magnitude, so its absolute error stays near 1e-7 however large the argument)
-__device__ __forceinline__ double log2_split(double z) {
-    int k;
-    const double m = frexp(z, &k);  // m in [0.5, 1)
-    return static_cast<double>(k) + static_cast<double>(log2f(static_cast<float>(m)));
-}
+// log2 of a positive finite number in double: it enters the normalisers of p and q, and the residual
+// max(0, p - q) sees the difference of their errors magnified by 1 / (its own mass); a few dozen calls
+// per batch row, so the cost does not show
+__device__ __forceinline__ double log2_split(double z) { return log2(z); }
 
 // End of a row epilogue (whole warp): everything the warp wrote for batch row b becomes visible
 // before the row's completion flag does.  The resample kernel polls the flag instead of waiting for
@@ -911,7 +942,7 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             ri.scale = scale;
             ri.lse2_p = lp_n;
             ri.lse2_q = lq_n;
-            P.info[b] = ri;
+            SPECKV_ST(P.info[b], ri);
         }
     }
     if (P.status && lane == 0) P.status[b] = status;
@@ -983,7 +1014,7 @@ __device__ __noinline__ void sample_epilogue(const KParams& P, int b, int gam, f
         ri.scale = scale;
         ri.lse2_p = lse2;
         ri.lse2_q = 0.0;
-        P.info[r] = ri;
+        SPECKV_ST(P.info[r], ri);
         P.out_tok[r] = (ok && greedy) ? amax : -1;
     }
     if (P.status && lane == 0) P.status[b] = status;
@@ -1008,7 +1039,7 @@ __device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, f
             ad = ldcg4(pd);
             for (int k = 1; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k), scale);
         }
-        out[G + 1 + lane] = ad;
+        SPECKV_ST(out[G + 1 + lane], ad);
     }
     if (lane <= G) {
         float4 at = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -1020,7 +1051,7 @@ __device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, f
                 if (idx != 0x7fffffff) at.y = __int_as_float(idx + P.v_begin);
             }
         }
-        out[lane] = at;
+        SPECKV_ST(out[lane], at);
     }
 }
 
@@ -1037,7 +1068,7 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid);
 // after the last sweep CTA has started and leaves most of the drain unused.
 // ----------------------------------------------------------------------------------------
 template <typename T, bool ALIGNED, int U>
-__global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __grid_constant__ KParams P) {
+__global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const __grid_constant__ KParams P) {
     if (static_cast<int>(blockIdx.x) >= P.n_sweep) {
         resample_body<T, ALIGNED>(P, static_cast<int>(blockIdx.x) - P.n_sweep);
         return;
@@ -1098,7 +1129,7 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
                 if (x >= 0 && x < P.V) {
                     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb +
                                     static_cast<long long>(pos) * P.tsp;
-                    P.tokl[static_cast<long long>(b) * P.G + pos] = make_float2(elem_to_float(row, x), elem_to_float(trow, x));
+                    SPECKV_ST(P.tokl[static_cast<long long>(b) * P.G + pos], make_float2(elem_to_float(row, x), elem_to_float(trow, x)));
                 }
             }
             part = sweep_warp<T, ALIGNED, PATH_DRAFT, U, STEP>(row, lo, hi, first, scale, sh_m0);
@@ -1121,7 +1152,7 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) sweep_kernel(const __gr
                 acc = (path == PATH_DRAFT) ? merge_draft(acc, o, scale)
                     : (path == PATH_TARGET) ? merge_target(acc, o) : merge_argmax(acc, o);
             }
-            P.part[static_cast<long long>(blockIdx.x)] = acc;
+            SPECKV_ST(P.part[static_cast<long long>(blockIdx.x)], acc);
         }
     } else if (row_ok || rem != 0 || warp != 0) {
         return;  // unused position: nothing to count; a flagged row keeps its first CTA for the epilogue
@@ -1201,7 +1232,7 @@ __device__ __forceinline__ uint4 rs_load4(const float* row, int e, int hi, float
     if (ALIGNED && e + 4 <= hi) return ldg_stream(row + e);
     float x[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) x[j] = (e + j < hi) ? row[e + j] : pad;
+    for (int j = 0; j < 4; ++j) x[j] = (e + j < hi) ? elem_to_float(row, e + j) : pad;
     return make_uint4(__float_as_uint(x[0]), __float_as_uint(x[1]), __float_as_uint(x[2]), __float_as_uint(x[3]));
 }
 template <typename T, bool ALIGNED>
@@ -1319,7 +1350,7 @@ __device__ __forceinline__ void rs_chunk_sums_mode(F make_const, const T* trow, 
 #pragma unroll
         for (int u = 0; u < KU; ++u) {
             const int ch = base + u * kWarps;
-            if (lane == 0 && ch < c1) csum[ch] = s[u];
+            if (lane == 0 && ch < c1) SPECKV_ST(csum[ch], s[u]);
         }
         if (next < c1) {
 #pragma unroll
@@ -1367,14 +1398,17 @@ constexpr int kRsStage = 2048;
 struct RsSums {
     const float* sh;    // staged copy, or nullptr
     const float* glob;
-    __device__ __forceinline__ float operator[](int ch) const { return sh ? sh[ch] : __ldcg(glob + ch); }
+    __device__ __forceinline__ float operator[](int ch) const {
+        if (sh) return sh[ch];
+        return dbg_ok(glob + ch, 4, DBG_WS_LOAD) ? __ldcg(glob + ch) : 0.f;
+    }
 };
 __device__ __forceinline__ RsSums rs_stage_sums(float* sh_cs, const float* csum, int nchunk) {
     RsSums r;
     r.glob = csum;
     r.sh = nullptr;
     if (nchunk <= kRsStage) {
-        for (int ch = threadIdx.x; ch < nchunk; ch += kThreads) sh_cs[ch] = __ldcg(csum + ch);
+        for (int ch = threadIdx.x; ch < nchunk; ch += kThreads) sh_cs[ch] = dbg_ok(csum + ch, 4, DBG_WS_LOAD) ? __ldcg(csum + ch) : 0.f;
         r.sh = sh_cs;
     }
     __syncthreads();

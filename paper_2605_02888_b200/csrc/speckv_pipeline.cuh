@@ -25,34 +25,20 @@
 
 namespace speckv {
 
-#ifndef SPECKV_PIPE_WARPS
-#define SPECKV_PIPE_WARPS 8
-#endif
-constexpr int kPipeWarps = SPECKV_PIPE_WARPS;        // consumer warps per CTA
+constexpr int kPipeWarpsCfg = 8;
+constexpr int kPipeWarps = kPipeWarpsCfg;        // consumer warps per CTA
 constexpr int kPipeThreads = (kPipeWarps + 2) * 32;  // + one producer warp + one epilogue warp
-#ifndef SPECKV_STAGE_GRAN
-#define SPECKV_STAGE_GRAN 1024                       // 16-byte granules per ring stage (16 KB)
-#endif
-#ifndef SPECKV_STAGES
-#define SPECKV_STAGES 6
-#endif
-#ifndef SPECKV_QUANTUM_STAGES
-#define SPECKV_QUANTUM_STAGES 16                     // target quantum: 256 KB
-#endif
-constexpr int kStageGran = SPECKV_STAGE_GRAN;
+constexpr int kStageGranCfg = 1024;  // 16-byte granules per ring stage (16 KB)
+constexpr int kStagesCfg = 6;
+constexpr int kQuantumStages = 16;  // target quantum: 256 KB
+constexpr int kStageGran = kStageGranCfg;
 constexpr int kStageBytes = kStageGran * 16;
-constexpr int kStages = SPECKV_STAGES;
-#ifndef SPECKV_SEG_SLOTS
-#define SPECKV_SEG_SLOTS 32
-#endif
-#ifndef SPECKV_PIPE_MAXB
-#define SPECKV_PIPE_MAXB 1024
-#endif
-#ifndef SPECKV_PIPE_CTAS
-#define SPECKV_PIPE_CTAS 2                           // CTAs per SM
-#endif
-constexpr int kSegSlots = SPECKV_SEG_SLOTS;          // segments between the consumers and the epilogue warp
-constexpr int kPipeMaxB = SPECKV_PIPE_MAXB;          // batch rows whose per-row tables fit the CTA
+constexpr int kStages = kStagesCfg;
+constexpr int kSegSlotsCfg = 32;
+constexpr int kPipeMaxBCfg = 1024;
+constexpr int kPipeCtasPerSm = 2;  // CTAs per SM
+constexpr int kSegSlots = kSegSlotsCfg;          // segments between the consumers and the epilogue warp
+constexpr int kPipeMaxB = kPipeMaxBCfg;          // batch rows whose per-row tables fit the CTA
 constexpr int kMaxSeg = 32;                          // partial slots per logit row
 constexpr int kWaitLimit = 1 << 22;
 
@@ -134,6 +120,11 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
 // global -> shared bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned); completion
 // is counted on `bar`.  No multicast: the destination is this CTA's own shared memory.
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+#ifdef SPECKV_DEBUG
+    // the consumers wait for these bytes, so a copy that fails the check is not dropped but redirected to
+    // the start of the draft logits (registered range 0), which is always there and large enough here
+    if (!dbg_ok(src, bytes, DBG_COPY)) src = reinterpret_cast<const void*>(g_dbg_ranges.lo[0]);
+#endif
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
                      smem_u32(dst)),
                  "l"(src), "r"(bytes), "r"(smem_u32(bar))
@@ -529,7 +520,7 @@ __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared&
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive(&sh.slot_free[slot]);
-                    P.part[si.part] = acc;
+                    SPECKV_ST(P.part[si.part], acc);
                     __threadfence();
                     const int total = si.jrows * (P.Lp / kStageGran);
                     if (atomicAdd(P.tick1 + si.b, si.stages) + si.stages == total) {  // row complete: enqueue it
@@ -565,7 +556,7 @@ __device__ __forceinline__ void pipe_epilogue_warp(const KParams& P, PipeShared&
 
 // ---- the kernel -------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(kPipeThreads, SPECKV_PIPE_CTAS) pipe_sweep_kernel(const __grid_constant__ KParams P) {
+__global__ void __launch_bounds__(kPipeThreads, kPipeCtasPerSm) pipe_sweep_kernel(const __grid_constant__ KParams P) {
     extern __shared__ __align__(128) unsigned char pipe_smem[];
     PipeShared& sh = *reinterpret_cast<PipeShared*>(pipe_smem);
     unsigned char* ring = pipe_smem + (sizeof(PipeShared) + 127) / 128 * 128;
@@ -615,7 +606,7 @@ __global__ void __launch_bounds__(kPipeThreads, SPECKV_PIPE_CTAS) pipe_sweep_ker
         const long long Lp = P.Lp;
         const long long Tg = static_cast<long long>(sh.prefix[P.B]) * Lp;
         const long long G = gridDim.x;
-        const long long qt = static_cast<long long>(SPECKV_QUANTUM_STAGES) * kStageGran;
+        const long long qt = static_cast<long long>(kQuantumStages) * kStageGran;
         long long K = (Tg + G * qt / 2) / (G * qt);  // quanta per CTA, rounded
         if (K < 1) K = 1;
         long long Q = (Tg + G * K - 1) / (G * K);

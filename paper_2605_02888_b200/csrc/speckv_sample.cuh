@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(kThreads, 4) sample_onepass_kernel(const __gri
                 z = warp_sumf(z);
                 second = bad ? __int_as_float(0x7fc00000) : z;
             }
-            if (lane == 0) cz[ch] = make_float2(mc, second);
+            if (lane == 0) SPECKV_ST(cz[ch], make_float2(mc, second));
         }
 #pragma unroll
         for (int u = 0; u < KU; ++u) cur[u] = nxt[u];

@@ -20,7 +20,7 @@ namespace speckv {
 // U loads of 16 bytes in flight per lane; the warp's merged state is the shard's state of that row.
 // No partials, no tickets.  (Wider slices use sweep_kernel with export_state set.)
 template <typename T, bool ALIGNED, int U>
-__global__ void __launch_bounds__(kThreads, SPECKV_MINB) shard_rows_kernel(const __grid_constant__ KParams P) {
+__global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) shard_rows_kernel(const __grid_constant__ KParams P) {
     const int lane = threadIdx.x & 31;
     const long long w = static_cast<long long>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
     if (w >= static_cast<long long>(P.B) * P.J) return;
@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(kThreads, SPECKV_MINB) shard_rows_kernel(const
                 const int x = __ldg(P.tok + static_cast<long long>(b) * P.G + pos) - P.v_begin;
                 if (x >= 0 && x < P.V) {
                     const T* trow = static_cast<const T*>(P.t) + static_cast<long long>(b) * P.tsb + static_cast<long long>(pos) * P.tsp;
-                    P.tokl[static_cast<long long>(b) * P.G + pos] = make_float2(elem_to_float(row, x), elem_to_float(trow, x));
+                    SPECKV_ST(P.tokl[static_cast<long long>(b) * P.G + pos], make_float2(elem_to_float(row, x), elem_to_float(trow, x)));
                 }
             }
             st = sweep_warp<T, ALIGNED, PATH_DRAFT, U, 32, false>(row, 0, P.V, lane, scale, nullptr);

@@ -177,6 +177,7 @@ constexpr int kSDynBytes = kSWarps * SStage<float>::kWarpBytes;
 static_assert(SStage<float>::kWarpBytes == SStage<__nv_bfloat16>::kWarpBytes, "one dynamic size for both types");
 
 __device__ __forceinline__ void cp_async16(uint32_t saddr, const void* g) {
+    if (!dbg_ok(g, 16, DBG_LOGIT16)) return;  // the slot keeps stale bytes: wrong numbers, counted, no fault
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(saddr), "l"(g) : "memory");
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -401,7 +402,7 @@ __device__ __noinline__ void s_resolve_stop(const KParams& P, const SParams& S, 
         ri.scale = static_cast<float>(kLog2e / static_cast<double>(Tf));
         ri.lse2_p = __ldcg(&pr->lse2_p);
         ri.lse2_q = n < gam ? __ldcg(&pr->lse2_q) : 0.0;
-        P.info[b] = ri;
+        SPECKV_ST(P.info[b], ri);
         __threadfence();
         const int at = atomicAdd(&S.ctrl->rs_tail, 1);
         asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(S.rsq + at), "r"(b + 1) : "memory");
@@ -540,7 +541,7 @@ __device__ __noinline__ void s_pair_epilogue(const KParams& P, const SParams& S,
     if (lane == 0) {
         PosRec r;
         r.H = Hi; r.c = ci; r.lse2_q = lse2_q; r.lse2_p = lse2_p; r.amax = amax; r.pad = 0;
-        S.pos[pair] = r;
+        SPECKV_ST(S.pos[pair], r);
         __threadfence();
         old = atomicOr(S.state + b, bits);
     }
@@ -604,7 +605,7 @@ __device__ __forceinline__ void s_warp_sums(const RsConst& c0, const T* trow, co
         }
 #pragma unroll
         for (int u = 0; u < KU; ++u)
-            if (lane == 0 && base + u < e) csum[base + u] = sm[u];
+            if (lane == 0 && base + u < e) SPECKV_ST(csum[base + u], sm[u]);
         if (base + KU < e) {
 #pragma unroll
             for (int u = 0; u < KU; ++u) {
@@ -701,7 +702,7 @@ __device__ __noinline__ void s_publish(const KParams& P, const SParams& S, const
     const int lane = threadIdx.x & 31;
     int t = 0;
     if (lane == 0) {
-        P.part[part_idx] = merged;
+        SPECKV_ST(P.part[part_idx], merged);
         __threadfence();
         t = atomicAdd(S.ptick + pair, 1);
     }

@@ -500,10 +500,30 @@ def test_empty_batch_and_argument_errors():
     w, s = _small()
     bt = gpu_batch(s)
     o = speckv.StepOutputs.allocate(bt)
-    o.workspace = o.workspace[:256]
-    with pytest.raises(speckv.SpeckvError) as e:
-        speckv.speckv_verify(bt, out=o)
-    assert e.value.code == 3
+    # the binding refuses buffers of the wrong size, shape or type before anything is launched
+    short = speckv.StepOutputs.allocate(bt)
+    short.workspace = short.workspace[:256]
+    with pytest.raises(ValueError, match="workspace"):
+        speckv.speckv_verify(bt, out=short)
+    bad = speckv.StepOutputs.allocate(bt)
+    bad.out_tokens = bad.out_tokens[:, :-1].contiguous()
+    with pytest.raises(ValueError, match="out_tokens"):
+        speckv.speckv_verify(bt, out=bad)
+    bad = speckv.StepOutputs.allocate(bt)
+    bad.H = bad.H.double()
+    with pytest.raises(TypeError, match="H"):
+        speckv.speckv_signals(bt, out=bad)
+    gm, _ = mlp_pair(synth.make_mlp(w, DEV))
+    with pytest.raises(ValueError, match="comp"):
+        speckv.speckv_step(bt, s["comp"][:, :1].contiguous(), gm)
+    with pytest.raises(ValueError, match="uniforms"):
+        speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],
+                     uniforms=s["uniforms"][:, :-1].contiguous())._c()
+    # the library's own check of a short workspace, through the C ABI
+    n = o.workspace.numel()
+    rc = speckv.load_library().speckv_verify(__import__("ctypes").byref(bt._c()), o.n_accepted.data_ptr(), o.out_tokens.data_ptr(),
+                                             o.row_status.data_ptr(), o.workspace.data_ptr(), n - 1, None)
+    assert rc == 3
 
 
 # ---- statistical properties of the CUDA path itself ----

@@ -412,3 +412,28 @@ def test_step_gives_flagged_rows_neutral_outputs():
         assert np.all(s["H"][b] == 0) and np.all(s["C"][b] == 0) and np.all(s["feat"][b] == 0)
     # the healthy row is untouched by its neighbours
     assert s["gamma_next"][0] in (2, 4, 6, 8) and s["feat"][0, 0] > 0 and s["out_tokens"][0, s["n_accepted"][0]] >= 0
+
+
+def test_residual_boundary_flags_relative_and_absolute():
+    # q = (0.6, 0.2, 0.2), p = (0.59, 0.2, 0.21) up to float32 rounding: token 0 is rejected with probability
+    # 1/60 and the residual, of mass W = 0.01, sits on token 2 alone, so every u' draws token 2 and no
+    # boundary is near.  With p = (0.59, 0.205, 0.205) the residual splits into two halves of 0.005:
+    # the boundary between tokens 1 and 2 lies at u' = 0.5.  A threshold 2e-5 * W away from it (2e-7 in units
+    # of probability) is outside the window on the normalised CDF but inside the absolute one; a threshold
+    # 0.1 * W away is outside both.
+    d = np.log(np.array([[[0.6, 0.2, 0.2]]])).astype(np.float32)
+    t = np.log(np.array([[[0.59, 0.205, 0.205], [1 / 3, 1 / 3, 1 / 3]]])).astype(np.float32)
+    p, q = _softmax(t[0, 0]), _softmax(d[0, 0])
+    w = np.maximum(0, p - q)
+    W = w.sum()
+    edge = w[1] / W
+    tok = np.zeros((1, 1), np.int32)
+    for du, want in ((2e-5, oracle.NEAR_CDF_ABS), (-2e-5, oracle.NEAR_CDF_ABS), (3e-7, oracle.NEAR_CDF), (0.1, 0)):
+        u = np.array([[[0.999, edge + du], [0.5, 0.5]]], np.float32)
+        r = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=tok, uniforms=u))
+        assert r["n_accepted"][0] == 0 and r["out_tokens"][0, 0] == (2 if du > 0 else 1)
+        assert r["near"][0] & (oracle.NEAR_CDF | oracle.NEAR_CDF_ABS) == want, (du, r["near"][0])
+    # a bonus draw (weights are probabilities, W = 1) never carries the absolute flag alone
+    u = np.array([[[0.0, 0.3], [0.5, 1 / 3 + 2e-5]]], np.float32)
+    r = oracle.verify(oracle.Batch(draft=d, target=t, draft_tokens=tok, uniforms=u))
+    assert r["n_accepted"][0] == 1 and not (r["near"][0] & oracle.NEAR_CDF_ABS)

@@ -3,19 +3,21 @@
 A serving process that has given all device memory to its framework's pool, or a plug-in that may
 only touch the buffers it is handed, cannot provide the workspace speckv_signals asks for.  The
 static variant carries its scratch inside the library image.  This file checks, through the C ABI,
-that it returns what speckv_signals returns, twice in a row on different inputs (the second call
-finds the first call's leftovers in the shared array), and that an over-sized batch is refused on
-the host.  It is named to be collected last, so a run that stops at the first failure has already
+that it returns what speckv_signals returns and what the CPU oracle computes, twice in a row on
+different inputs (the second call finds the first call's leftovers in the shared array), that the
+device's free memory is the same after the calls as before them, and that an over-sized batch is
+refused on the host.  It is named to be collected last, so a run that stops at the first failure has already
 run every other test."""
 import ctypes as C
 
 import pytest
 import torch
 
+import oracle
 import paper_2605_02888_b200 as speckv
 from paper_2605_02888_b200 import binding, synth
 
-from parity import ATOL, RTOL, close, gpu_batch
+from parity import ATOL, RTOL, close, gpu_batch, oracle_batch
 
 DEV = "cuda:0"
 
@@ -33,13 +35,19 @@ def test_static_scratch_matches_workspace_variant_on_two_calls_in_a_row():
         bt = gpu_batch(s)
         assert speckv.workspace_size(bt) <= binding.STATIC_SCRATCH_BYTES
         ref = {k: v.clone() for k, v in speckv.speckv_signals(bt).items()}
+        want = oracle.signals(oracle_batch(s))  # the oracle's signals read the draft rows only
         for t in outs.values():
             t.fill_(-7)                         # stale contents must be overwritten
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         got = speckv.speckv_signals_static(bt, **outs)
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
         assert torch.equal(got["row_status"], ref["row_status"])
+        assert (got["row_status"].cpu().numpy() == want["row_status"]).all()
         for k in ("H", "C", "feat"):
-            close(got[k].cpu().numpy(), ref[k].cpu().numpy(), f"{k} (call {step})", rtol=RTOL, atol=ATOL)
+            close(got[k].cpu().numpy(), ref[k].cpu().numpy(), f"{k} against speckv_signals (call {step})", rtol=RTOL, atol=ATOL)
+            close(got[k].cpu().numpy(), want[k], f"{k} against the oracle (call {step})", rtol=RTOL, atol=ATOL)
 
 
 def test_static_scratch_limit_is_checked_on_the_host():
