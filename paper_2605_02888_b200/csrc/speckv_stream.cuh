@@ -156,6 +156,8 @@ struct SShared {
     unsigned short pre[kSMaxPhase][kSMaxB / 32 + 1];
     unsigned char gam[kSMaxB];
     int job_head, job_tail;
+    unsigned long long wake;  // mbarrier the idle warps sleep on; whoever adds work to the ring or the queue arrives on it
+    int wake_gen;             // arrivals so far (the parity an idle warp waits for)
     SJob jobs[kSJobs];
     SItem ring[kSRing];
 };
@@ -744,6 +746,8 @@ __device__ __forceinline__ void s_job_push(const KParams& P, const SParams& S, S
             e->pair = j.pair; e->pair_total = j.pair_total; e->Tf = j.Tf;
             __threadfence_block();
             *reinterpret_cast<volatile int*>(&e->ready) = at + 1;
+            atomicAdd(&sh.wake_gen, 1);
+            mbar_arrive(&sh.wake);
         }
     }
     at = __shfl_sync(0xffffffffu, at, 0);
@@ -844,6 +848,24 @@ __device__ __forceinline__ void s_resample_job(const KParams& P, const SParams& 
     }
 }
 
+// Idle warps do not spin: they block on an mbarrier phase (the hardware parks the warp) until somebody
+// has added work, or for about two microseconds at most.
+__device__ __forceinline__ void s_wake(SShared& sh) {
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&sh.wake_gen, 1);
+        mbar_arrive(&sh.wake);
+    }
+}
+__device__ __forceinline__ void s_nap(SShared& sh, int gen) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(smem_u32(&sh.wake)), "r"(static_cast<uint32_t>(gen & 1)), "r"(2000u)
+        : "memory");
+    (void)ok;
+}
+
 // One step of filling, by whichever warp gets the lock: a resample share if one is waiting (its rows
 // are the freshest in L2), else the next item of the stream.
 // `starving`: the caller has nothing to do until the ring grows (it may sleep a little); otherwise it
@@ -854,7 +876,7 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
     int got = 0;
     if (lane == 0) got = (atomicCAS(&sh.lock, 0, 1) == 0);
     got = __shfl_sync(0xffffffffu, got, 0);
-    if (!got) { if (starving) __nanosleep(1500); return; }
+    if (!got) return;
     auto unlock = [&]() {
         __syncwarp();
         if (lane == 0) { __threadfence_block(); atomicExch(&sh.lock, 0); }
@@ -862,7 +884,7 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
     const int tail = s_vol(&sh.tail);
     SItem& it = sh.ring[tail % kSRing];
     const bool slot_free = tail < kSRing || s_vol(&it.busy) == 0;
-    if (!slot_free || s_vol(&sh.exhausted)) { unlock(); if (starving) __nanosleep(1500); return; }
+    if (!slot_free || s_vol(&sh.exhausted)) { unlock(); return; }
 
     // A share of a queued draw comes first (its rows are the freshest in L2).  The counter is a plain
     // atomic add, so nobody retries; a share number beyond the rows queued so far (another CTA was quicker)
@@ -909,6 +931,7 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
             *reinterpret_cast<volatile int*>(&sh.tail) = tail + 1;
         }
         unlock();
+        s_wake(sh);
         return;
     }
 
@@ -971,6 +994,7 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
             }
         }
         unlock();
+        if (k > 0) s_wake(sh);
         return;
     }
 
@@ -980,7 +1004,7 @@ __device__ __noinline__ void s_try_fill(const KParams& P, const SParams& S, SSha
         else if (++sh.idle_polls > S.poll_limit) { sh.error = 1; sh.exhausted = 1; }
     }
     unlock();
-    if (starving) __nanosleep(1500);
+    if (sh.exhausted) s_wake(sh);
 }
 
 // Claims the next quantum of the CTA's ring for this warp: one atomic add on the item's counter, which
@@ -994,6 +1018,7 @@ __device__ __forceinline__ bool s_claim(const KParams& P, const SParams& S, SSha
                                         int& out_q, bool blocking) {
     const int lane = threadIdx.x & 31;
     for (;;) {
+        const int gen = s_vol(&sh.wake_gen);  // read before looking for work: work added after this ends the nap at once
         if (blocking) {  // a warp without a quantum in hand takes queued bookkeeping first
             const int r = s_job_reserve(sh);
             if (r >= 0) { s_job_run<T>(P, S, sh, r); continue; }
@@ -1001,7 +1026,9 @@ __device__ __forceinline__ bool s_claim(const KParams& P, const SParams& S, SSha
         if (cursor >= s_vol(&sh.tail)) {
             if (!blocking) return false;
             if (s_vol(&sh.exhausted)) return false;
+            const int before = s_vol(&sh.tail);
             s_try_fill<T>(P, S, sh, true);
+            if (s_vol(&sh.tail) == before && !s_vol(&sh.exhausted)) s_nap(sh, gen);  // nothing came of it
             continue;
         }
         SItem* it = &sh.ring[cursor % kSRing];
@@ -1040,7 +1067,9 @@ __global__ void __launch_bounds__(kSThreads, 1) stream_kernel(const __grid_const
     if (threadIdx.x == 0) {
         sh.tail = 0; sh.lock = 0; sh.exhausted = 0; sh.stream_done = 0; sh.error = 0;
         sh.idle_polls = 0; sh.first_taken = 0; sh.n_blk = n_blk;
-        sh.job_head = 0; sh.job_tail = 0; sh.pend_share = -1;
+        sh.job_head = 0; sh.job_tail = 0; sh.pend_share = -1; sh.wake_gen = 0;
+        mbar_init(&sh.wake, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x < kSJobs) sh.jobs[threadIdx.x].ready = 0;  // shared memory keeps what the last launch left
     for (int blk = warp; blk < n_blk; blk += kSWarps) {
