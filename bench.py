@@ -350,7 +350,7 @@ def main():
         clocks["ms_per_step_x_sm_mhz"] = ms_step * clocks["sm_mhz"]
 
     # dominant kernel alone: events recorded by the library around the sweep kernel
-    n_prof = min(args.steps, 200)
+    n_prof = min(max(args.steps, 100), 200)
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n_prof)]
     for i in range(n_prof):
         one(i, events=evs[i])
@@ -375,6 +375,7 @@ def main():
                 "kernel_ms_min": min(sweep_ms),
                 "kernel_covers": "sweep + row epilogues + fresh-token draw" if one_launch else "sweep + row epilogues",
                 "resample_kernel_ms": None if one_launch else sum(resample_ms) / n_prof,
+                "kernel_ms_median": statistics.median(sweep_ms),
                 "timed_over": f"{n_prof} steps after the timed region, CUDA events recorded inside the library call",
                 "frac_of_8TBps": achieved / 8000.0,
                 "step_GBps": sum(bytes_step[i % n_batches] for i in range(args.steps)) / args.steps / (ms_step * 1e-3) / 1e9}
