@@ -436,14 +436,16 @@ def test_full_size_step_repeats_bit_for_bit_with_one_workspace():
                                again[k].view(torch.int32) if again[k].dtype == torch.float32 else again[k]), k
 
 
-@pytest.mark.parametrize("name,B,V", [("b256", 64, 32000), ("b512_mixed", 400, 8000), ("b512_mixed", 32, 8000)])
-def test_step_can_be_captured_in_a_cuda_graph(name, B, V):
+@pytest.mark.parametrize("name,B,V,flags", [("b256", 64, 32000, 0), ("b512_mixed", 400, 8000, 0), ("b512_mixed", 32, 8000, 0),
+                                            ("b256", 64, 32000, 2)])
+def test_step_can_be_captured_in_a_cuda_graph(name, B, V, flags):
     # the library only enqueues work on the caller's stream (no allocation, no synchronisation), so a step
-    # can be recorded once and replayed: single-launch path, ring sweep + dependent resample kernel, fp32 fallback
+    # can be recorded once and replayed: single-launch path, ring sweep + dependent resample kernel, fp32 fallback,
+    # and the stream kernel (flags = 2, SPECKV_SCHEDULE_STREAM)
     w = synth.scaled(synth.WORKLOADS[name], B=B, V=V)
     s = synth.make_step(w, 0, DEV)
     gm, _ = mlp_pair(synth.make_mlp(w, DEV))
-    bt = gpu_batch(s)
+    bt = gpu_batch(s, flags=flags)
     out = speckv.StepOutputs.allocate(bt, gm.n_out)
     direct = {k: v.clone() for k, v in speckv.speckv_step(bt, s["comp"], gm, out=out).items()}
     torch.cuda.synchronize()

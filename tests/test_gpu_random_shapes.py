@@ -9,7 +9,7 @@ import torch
 
 import oracle
 import paper_2605_02888_b200 as speckv
-from paper_2605_02888_b200 import synth, vocab_shard
+from paper_2605_02888_b200 import binding, synth, vocab_shard
 
 from parity import compare_step, gpu_batch, mlp_pair, oracle_batch
 
@@ -38,6 +38,11 @@ def test_random_shapes(seed):
             out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
             torch.cuda.synchronize()
             compare_step(out, ref)
+        if (V * (2 if dtype == "bf16" else 4)) % 16 == 0:   # rows of whole 16-byte granules: the stream kernel takes them
+            for flags in (binding.SCHEDULE_STREAM, binding.SCHEDULE_STREAM | binding.READ_ALL_TARGET_ROWS):
+                out = speckv.speckv_step(gpu_batch(s, flags=flags), s["comp"], gm)
+                torch.cuda.synchronize()
+                compare_step(out, ref)
         if V >= 64 and rnd.random() < 0.4:
             n_shards = rnd.choice([2, 3, 4])
             out = vocab_shard.step_emulated(gpu_batch(s), n_shards, s["comp"], gm)
@@ -95,6 +100,10 @@ def test_random_edge_inputs(seed):
         out = speckv.speckv_step(gpu_batch(s), s["comp"], gm)
         torch.cuda.synchronize()
         compare_step(out, ref)
+        if (V * (2 if dtype == "bf16" else 4)) % 16 == 0:
+            out = speckv.speckv_step(gpu_batch(s, flags=binding.SCHEDULE_STREAM), s["comp"], gm)
+            torch.cuda.synchronize()
+            compare_step(out, ref)
         if V >= 1000:
             out = vocab_shard.step_emulated(gpu_batch(s), rnd.choice([2, 3]), s["comp"], gm)
             torch.cuda.synchronize()
