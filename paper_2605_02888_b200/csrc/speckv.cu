@@ -90,6 +90,7 @@ int choose_nsplit(int B, int J, int V, speckv_dtype dt) {
     return ns;
 }
 
+constexpr int kEarlyPositions = 2;   // positions whose acceptance tests the sliced sweep takes ahead of the rest of the row
 constexpr int kRsChunksPerCta = 64;  // 256-element chunks of the stop position that one resample CTA sums
 
 Plan make_plan(const speckv_batch* bt) {
@@ -103,7 +104,7 @@ Plan make_plan(const speckv_batch* bt) {
     if (p.R < 1) p.R = 1;
     p.chunks_per_cta = (p.nchunk + p.R - 1) / p.R;
     size_t off = 0;
-    p.off_tick = off; off = align_up(off + (4 * B + 4) * sizeof(int));  // tickets, counters, row queue, row flags
+    p.off_tick = off; off = align_up(off + (6 * B + 4) * sizeof(int));  // tickets, counters, row queue, row flags, first-generation tickets, early stops
     p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
     p.off_part = off; off = align_up(off + B * p.J_full * kMaxSplit * sizeof(float4));
     p.off_csum = off; off = align_up(off + B * p.nchunk * sizeof(float));
@@ -426,7 +427,7 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
         }
     }
 
-    if (cudaMemsetAsync(P.tick1, 0, (4 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
+    if (cudaMemsetAsync(P.tick1, 0, (6 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;
 
     // the staged sweep wants whole 16-byte granules per row and a batch its per-row tables can hold
@@ -445,6 +446,15 @@ constexpr int kPipeMinB = 384;
     // everything is done and a flag would only cost it a round trip
     P.rdone = (verify && !staged) ? P.rowq + P.B : nullptr;
     P.tokl = (verify && !staged) ? reinterpret_cast<float2*>(static_cast<char*>(ws) + pl.off_tokl) : nullptr;
+    if (verify && !staged) {
+        // generation order: positions 0..k of every batch row first, so that their acceptance tests are in
+        // before the CTAs of the later target rows start (most walks that stop early stop at the first two
+        // positions, and a later position's test would come too late for the CTAs behind it anyway)
+        P.k_early = P.G >= 2 ? kEarlyPositions - 1 : 0;
+        P.read_all = (bt->flags & SPECKV_READ_ALL_TARGET_ROWS) ? 1 : 0;
+        P.tick_early = P.rowq + 2 * P.B;
+        P.early = P.rowq + 3 * P.B;
+    }
     P.rs_reverse = staged ? 1 : 0;  // the ring sweep ends all at once: no drain for the resample kernel to fill
     P.Lg = static_cast<int>(row_bytes / 16);
     P.Lp = (P.Lg + kStageGran - 1) / kStageGran * kStageGran;

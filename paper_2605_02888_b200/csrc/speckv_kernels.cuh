@@ -83,6 +83,12 @@ struct KParams {
     int sample;  // 1: draft-side sampling (every drafted position draws a token from its own row)
     int rs_tail, R2, chunks_per_cta2;  // resample: the last rs_tail draws in launch order use R2 CTAs each
     int wait_limit;  // polls a resample CTA spends on its row's completion flag before it gives the row up
+    // Generation order of the sweep grid (verification, early != nullptr): first the draft and target rows of
+    // positions 0..k_early of every batch row, then the remaining draft rows, last the remaining target rows,
+    // which are left unread where the walk is already known to have stopped at a position <= k_early.
+    int k_early, read_all;
+    int* early;       // [B] 0 = not known yet, else stop position + 1, or G + 2 when the walk passes k_early
+    int* tick_early;  // [B] arrivals of the first generation's CTAs
     int rs_reverse;  // resample kernel: 1 = last batch row first (after a sweep it cannot overlap: those rows are the freshest in L2)
     int Lg, Lp;  // staged sweep: 16-byte granules per logit row, and the same padded to whole ring stages
     const void* d; long long dsb, dsp;
@@ -790,30 +796,34 @@ __device__ __forceinline__ int row_done_wait(const int* flag, int limit) {
     return 0;
 }
 
-// Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
-// merges the nd partials at pd (draft position i) and the nt partials at pt (target position i).
-// gam and Tf are the row's gamma and temperature as the sweep read them.  Everything the row
-// needs from memory that does not depend on other loads is requested first, so the epilogue
-// costs one memory round trip (two when the sweep did not leave the logits at the draft tokens).
-// Order: what the resample kernel needs (acceptance, stop position, normalisers), the row's
-// completion flag, then the signals and the controller.
+// What one lane of a row's epilogue learns about its position (lane i: draft position i, target position i).
+struct RowDecide {
+    int x;            // draft token (-1 where the lane has none)
+    float u_res;      // second uniform of the position
+    float Hi, ci;     // entropy (nats) and confidence of the draft distribution
+    double lse2_q, lse2_p;  // log2-normalisers of draft and target
+    int amax;         // greedy rows: argmax of the target row
+    bool dbad, tbad;  // non-finite draft row / target row at this position
+    bool badtok, accept, any_dbad;
+};
+
+// The per-position part of the row epilogue: lane i < n_lanes merges the nd partials at pd (draft position
+// i) and the nt partials at pt (target position i) and takes the acceptance test of its position.  One
+// compiled body serves the row epilogue and the prefix epilogue below, so that both reach the same bits.
 template <typename T>
-__device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd, int nd,
-                                          const float4* pt, int nt) {
+__device__ __noinline__ void row_decide(const KParams& P, int b, int gam, float Tf, int status, int n_lanes,
+                                        const float4* pd, int nd, const float4* pt, int nt, RowDecide& o) {
     const int lane = threadIdx.x & 31;
     const int G = P.G;
     const bool verify = (P.mode & MODE_VERIFY) != 0;
     constexpr int kPre = 4;  // partials fetched ahead per lane; more are rare
-
-    int status = 0;
-    if (gam < 1 || gam > G) status |= 1;
-    if (!(Tf >= 0.f) || Tf == __int_as_float(0x7f800000)) status |= 8;
     const bool greedy = (Tf == 0.f);
     const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
     const double sd = static_cast<double>(scale);
-    const bool dr_on = !status && lane < gam;
-    const bool tg_on = !status && verify && lane <= gam;
-    const bool tok_on = !status && verify && lane < gam;
+    const bool in = lane < n_lanes;
+    const bool dr_on = in && !status && lane < gam;
+    const bool tg_on = in && !status && verify && lane <= gam;
+    const bool tok_on = in && !status && verify && lane < gam;
 
     // ---- first round trip ----
     const long long ps = P.part_stride > 0 ? P.part_stride : 1;  // partials of a logit row: adjacent, or one per shard
@@ -836,8 +846,6 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             at += (x > 0 ? min(x / P.shard_width, P.n_shards - 1) : 0) * P.tokl_stride;
         tl = __ldcg(P.tokl + at);
     }
-    CtlRegs ctl;
-    if ((P.mode & MODE_MLP) && !status) ctl = ctl_load(P, b, lane);
 
     const bool badtok = tok_on && (x < 0 || x >= P.V);
     float dxf = tl.x, txf = tl.y;
@@ -864,8 +872,11 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             if (k < nd) ad = merge_draft(ad, qd[k], scale);
             if (k < nt) at = greedy ? merge_argmax(at, qt[k]) : merge_target(at, qt[k]);
         }
-        for (int k = kPre; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k * ps), scale);
-        for (int k = kPre; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k * ps)) : merge_target(at, ldcg4(pt + k * ps));
+        // (only lanes that have a position: the partials of the others would lie outside the array)
+        if (dr_on)
+            for (int k = kPre; k < nd; ++k) ad = merge_draft(ad, ldcg4(pd + k * ps), scale);
+        if (tg_on)
+            for (int k = kPre; k < nt; ++k) at = greedy ? merge_argmax(at, ldcg4(pt + k * ps)) : merge_target(at, ldcg4(pt + k * ps));
         if (dr_on) {
             const float m = ad.x, cnt = ad.y, Zx = ad.z, S = ad.w;
             const float Z = cnt + Zx;
@@ -892,8 +903,6 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
         any_dbad = __any_sync(0xffffffffu, dbad);
     }
 
-    // Acceptance first: the resample kernel waits for this row's stop position, nothing waits for
-    // the signals and the controller, which follow the completion flag.
     if (status == 0 && !any_dbad && tok_on && !badtok && !tbad) {
         if (greedy) {
             accept = (x == amax);
@@ -905,6 +914,60 @@ __device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, floa
             accept = (l2u + lq) < lp;
         }
     }
+    o.x = x; o.u_res = u_res; o.Hi = Hi; o.ci = ci; o.lse2_q = lse2_q; o.lse2_p = lse2_p; o.amax = amax;
+    o.dbad = dbad; o.tbad = tbad; o.badtok = badtok; o.accept = accept; o.any_dbad = any_dbad;
+}
+
+// Prefix epilogue (one warp): run when the partials of a batch row's first positions 0..k are in, while
+// the rest of the row is still being swept.  It takes the acceptance tests of those positions and
+// publishes where the walk stops if it stops there, so that CTAs which have not started yet can leave
+// target rows behind that position unread.  early[b] = stop position + 1, or G + 2 when the walk passes k.
+template <typename T>
+__device__ __noinline__ void prefix_epilogue(const KParams& P, int b, int gam, float Tf) {
+    const int lane = threadIdx.x & 31;
+    const long long row0 = static_cast<long long>(b) * P.J;
+    RowDecide d;
+    row_decide<T>(P, b, gam, Tf, 0, P.k_early + 1, P.part + (row0 + P.G + 1 + lane) * P.nsplit, P.nsplit,
+                  P.part + (row0 + lane) * P.nsplit, P.nsplit, d);
+    const bool in = lane <= P.k_early && lane <= gam;
+    const unsigned stop = __ballot_sync(0xffffffffu, in && (d.tbad || d.dbad || (lane < gam && (d.badtok || !d.accept))));
+    if (lane == 0) {
+        const int e = stop ? __ffs(stop) : P.G + 2;
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(P.early + b), "r"(e) : "memory");
+    }
+}
+
+// Row epilogue: one warp, run by whoever learns that all partials of batch row b are in.  Lane i
+// merges the nd partials at pd (draft position i) and the nt partials at pt (target position i).
+// gam and Tf are the row's gamma and temperature as the sweep read them.  Everything the row
+// needs from memory that does not depend on other loads is requested first, so the epilogue
+// costs one memory round trip (two when the sweep did not leave the logits at the draft tokens).
+// Order: what the resample kernel needs (acceptance, stop position, normalisers), the row's
+// completion flag, then the signals and the controller.
+template <typename T>
+__device__ __noinline__ void row_epilogue(const KParams& P, int b, int gam, float Tf, const float4* pd, int nd,
+                                          const float4* pt, int nt) {
+    const int lane = threadIdx.x & 31;
+    const int G = P.G;
+    const bool verify = (P.mode & MODE_VERIFY) != 0;
+
+    int status = 0;
+    if (gam < 1 || gam > G) status |= 1;
+    if (!(Tf >= 0.f) || Tf == __int_as_float(0x7f800000)) status |= 8;
+    const bool greedy = (Tf == 0.f);
+    const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
+    const bool tg_on = !status && verify && lane <= gam;
+
+    CtlRegs ctl;
+    if ((P.mode & MODE_MLP) && !status) ctl = ctl_load(P, b, lane);
+    RowDecide dec;
+    row_decide<T>(P, b, gam, Tf, status, 32, pd, nd, pt, nt, dec);
+    const int x = dec.x;
+    const float u_res = dec.u_res, Hi = dec.Hi, ci = dec.ci;
+    const double lse2_q = dec.lse2_q, lse2_p = dec.lse2_p;
+    const int amax = dec.amax;
+    const bool tbad = dec.tbad, badtok = dec.badtok, accept = dec.accept, any_dbad = dec.any_dbad;
+
     // The positions are walked in order; the walk ends at the first one whose target row is non-finite
     // (which flags the row), whose draft token is out of range, or whose token is rejected.  Target rows
     // behind that position are not part of the step (Sec. 3.1 discards what follows the first mismatch):
@@ -1058,6 +1121,9 @@ __device__ __noinline__ void export_epilogue(const KParams& P, int b, int gam, f
 // One CTA's share of a batch row's fresh-token draw (defined with the resample kernel below).
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ void resample_body(const KParams& P, const int bid);
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void resample_row(const KParams& P, const int b, const int r, const int mode, const int n,
+                                             const int4 lo4, const int4 hi4, const int share, const int Rr, const int cpc);
 
 // ----------------------------------------------------------------------------------------
 // Sweep kernel.  CTAs 0 .. n_sweep-1 sweep one slice of one logit row each.  With verification the
@@ -1075,22 +1141,56 @@ __global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const 
     }
     __shared__ float4 sh_part[kWarps];
     __shared__ int sh_count;
+    __shared__ int sh_early;
     __shared__ float sh_m0[kWarps];
     asm volatile("griddepcontrol.launch_dependents;");  // a dependent resample kernel may be scheduled as SMs free up
-    if (threadIdx.x == 0) sh_count = 0;
-    if (threadIdx.x < kWarps) sh_m0[threadIdx.x] = kFloor;
-    __syncthreads();  // before any load is issued
-
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int per_row = P.J * P.nsplit;
-    const int b = blockIdx.x / per_row;
-    const int rem = blockIdx.x - b * per_row;
-    const int j = rem / P.nsplit;
-    const int s = rem - j * P.nsplit;
     const bool verify = (P.mode & MODE_VERIFY) != 0;
-
+    int b, j, s, gen = 0;
+    if (P.early) {
+        // generation order: CTAs start in index order, so a later generation starts when the earlier ones
+        // are all under way and, for all but the smallest batches, long after the first one has finished
+        const int ns = P.nsplit, k1 = P.k_early + 1;
+        const int nA = k1 * P.B * 2 * ns, nB = (P.G - k1) * P.B * ns;
+        int i = blockIdx.x, p, is_draft;
+        if (i < nA) {
+            p = i / (2 * P.B * ns); i -= p * (2 * P.B * ns);
+            b = i / (2 * ns); i -= b * (2 * ns);
+            is_draft = i / ns; s = i - is_draft * ns;
+        } else {
+            // the later generations go batch row by batch row, so that the rows complete one after another
+            gen = (i < nA + nB) ? 1 : 2;
+            i -= (gen == 1) ? nA : nA + nB;
+            const int per_b = (gen == 1 ? P.G - k1 : P.G + 1 - k1) * ns;
+            b = i / per_b; i -= b * per_b;
+            p = i / ns; s = i - p * ns;
+            p += k1;
+            is_draft = (gen == 1);
+        }
+        j = is_draft ? P.G + 1 + p : p;
+    } else {
+        const int per_row = P.J * P.nsplit;
+        b = blockIdx.x / per_row;
+        const int r = blockIdx.x - b * per_row;
+        j = r / P.nsplit;
+        s = r - j * P.nsplit;
+    }
+    // the row's gamma and temperature travel together with the one thing a CTA of the last generation has
+    // to learn first: one memory round trip before the CTA knows whether it has work
     int gam = P.gamma ? P.gamma[b] : P.G;
     float Tf = P.temp ? P.temp[b] : P.temp_scalar;
+    if (threadIdx.x == 0) {
+        sh_count = 0;
+        // one thread reads what is known of the row's stop position, so that the whole CTA takes one decision
+        int e = 0;
+        if (gen == 2 && !P.read_all)
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(e) : "l"(P.early + b) : "memory");
+        sh_early = e;
+    }
+    if (threadIdx.x < kWarps) sh_m0[threadIdx.x] = kFloor;
+    __syncthreads();  // before any load is issued
+    const int rem = j * P.nsplit + s;
+
     const bool row_ok = (gam >= 1 && gam <= P.G) && (Tf >= 0.f) && (Tf != __int_as_float(0x7f800000));
     const bool greedy = (Tf == 0.f);
     const float scale = static_cast<float>(kLog2e / static_cast<double>(greedy ? 1.f : Tf));
@@ -1102,8 +1202,17 @@ __global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const 
     const bool is_target = P.sample || (verify && j <= P.G);
     const int pos = is_target ? j : (verify ? j - (P.G + 1) : j);
     const bool active = row_ok && ((is_target && !P.sample) ? pos <= gam : pos < gam);
+    const long long pidx = (static_cast<long long>(b) * P.J + j) * P.nsplit + s;  // this CTA's partial
 
-    if (active) {
+    // the walk stopped at a position before this one
+    const bool skipped = active && gen == 2 && sh_early != 0 && sh_early <= P.k_early + 1;
+    if (skipped) {
+        // the row epilogue never looks behind the stop position; the partial only has to be finite
+        if (warp != 0) return;
+        if (lane == 0)
+            SPECKV_ST(P.part[pidx], greedy ? make_float4(kFloor, __int_as_float(0x7fffffff), 0.f, 0.f)
+                                           : make_float4(kFloor, 0.f, 0.f, 0.f));
+    } else if (active) {
         // the CTA's slice of the row
         const int v0 = s * P.per_split;
         const int v1 = min(P.nvec, v0 + P.per_split);
@@ -1152,7 +1261,20 @@ __global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const 
                 acc = (path == PATH_DRAFT) ? merge_draft(acc, o, scale)
                     : (path == PATH_TARGET) ? merge_target(acc, o) : merge_argmax(acc, o);
             }
-            SPECKV_ST(P.part[static_cast<long long>(blockIdx.x)], acc);
+            SPECKV_ST(P.part[pidx], acc);
+        }
+        if (P.early && gen == 0) {
+            // first generation: the last of the row's CTAs of positions 0..k_early takes their acceptance tests
+            const int n_pre = (min(P.k_early, gam) + 1 + min(P.k_early + 1, gam)) * P.nsplit;
+            int last_pre = 0;
+            if (lane == 0) {
+                __threadfence();
+                last_pre = (atomicAdd(P.tick_early + b, 1) == n_pre - 1);
+            }
+            if (__shfl_sync(0xffffffffu, last_pre, 0)) {
+                __threadfence();
+                prefix_epilogue<T>(P, b, gam, Tf);
+            }
         }
     } else if (row_ok || rem != 0 || warp != 0) {
         return;  // unused position: nothing to count; a flagged row keeps its first CTA for the epilogue
@@ -1161,6 +1283,7 @@ __global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const 
     // ticket: the last of the row's active CTAs runs the row epilogue; nobody waits
     const int n_rows = P.sample ? gam : (verify ? 2 * gam + 1 : gam);
     const int n_tickets = row_ok ? n_rows * P.nsplit : 1;
+    const long long row0 = static_cast<long long>(b) * P.J;
     int last_row = 0;
     if (lane == 0) {
         __threadfence();
@@ -1168,7 +1291,6 @@ __global__ void __launch_bounds__(kThreads, kSweepCtasPerSm) sweep_kernel(const 
     }
     if (!__shfl_sync(0xffffffffu, last_row, 0)) return;
     __threadfence();
-    const long long row0 = static_cast<long long>(b) * P.J;
     if (P.sample) {
         sample_epilogue(P, b, gam, Tf, P.part + (row0 + lane) * P.nsplit, P.nsplit);
         return;
@@ -1503,8 +1625,6 @@ __device__ __forceinline__ int rs_search(const RsConst& c, const T* trow, const 
 template <typename T, bool ALIGNED>
 __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     __shared__ int sh_flag;
-    __shared__ int sh_empty;
-    __shared__ float sh_cs[kRsStage];
     // one-dimensional grid, R consecutive CTAs per batch row: the CTAs of a row are neighbours in
     // launch order, so rows finish one after the other and their searches overlap the other rows' sums
     // (draft-side sampling: one draw per drafted position; r counts positions, b = r / gamma_max)
@@ -1516,7 +1636,7 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
     const int Rr = tail ? P.R2 : P.R;
     const int cpc = tail ? P.chunks_per_cta2 : P.chunks_per_cta;
     const int bq = tail ? (n_all - P.rs_tail) + (bid - n_head) / Rr : bid / Rr;
-    const int share = tail ? (bid - n_head) % Rr : bid - bq * Rr;
+    const int share = tail ? (bid - n_head) % Rr : bid % Rr;
     const int r = P.rs_reverse ? (P.sample ? P.B * P.G : P.B) - 1 - bq : bq;
     const int b = P.sample ? r / P.G : r;
     // Launched as a programmatic dependent of the sweep kernel, so its CTAs become resident as the
@@ -1559,6 +1679,18 @@ __device__ __forceinline__ void resample_body(const KParams& P, const int bid) {
         mode = lo4.x;
         n = lo4.y;
     }
+    resample_row<T, ALIGNED>(P, b, r, mode, n, lo4, hi4, share, Rr, cpc);
+}
+
+// One CTA's share (chunks share*cpc ...) of draw r of batch row b; the last of the draw's Rr CTAs to arrive
+// locates the token.  lo4 / hi4: the row's record as loaded from P.info[r].
+template <typename T, bool ALIGNED>
+__device__ __forceinline__ void resample_row(const KParams& P, const int b, const int r, const int mode, const int n,
+                                             const int4 lo4, const int4 hi4, const int share, const int Rr, const int cpc) {
+    __shared__ int sh_flag;
+    __shared__ int sh_empty;
+    __shared__ float sh_cs[kRsStage];
+    const int4* ip = reinterpret_cast<const int4*>(P.info + r);
     if (mode == RS_NONE) return;  // greedy or flagged row: nothing to draw
     const long long out_at = P.sample ? static_cast<long long>(r) : static_cast<long long>(b) * (P.G + 1) + n;
 

@@ -68,6 +68,13 @@ def test_no_access_leaves_its_buffers(debug_library):
             if V % 8 == 0:
                 _check(w, flags=binding.SCHEDULE_STREAM)
     assert _violations(L)[0] == 0, _violations(L)
+    # a single batch row cut into many slices: more partials per logit row than the epilogue fetches ahead,
+    # and nothing behind the row's partials but the end of the array
+    for dtype, V, G in (("fp32", 32000, 8), ("bf16", 128256, 2)):
+        w = synth.Workload("d", B=1, gamma_max=G, V=V, dtype=dtype, gamma_mode="fixed", gamma_fixed=G, temperature=0.5,
+                           sigma_d=(0.6,), seed=50)
+        _check(w)
+    assert _violations(L)[0] == 0, _violations(L)
     # the stream kernel with several slices per row, and with more than 32 quanta per item
     for dtype, V in (("bf16", 300000), ("fp32", 40000)):
         w = synth.Workload("d", B=6, gamma_max=3, V=V, dtype=dtype, gamma_mode="ragged", temperature=0.8,
