@@ -371,7 +371,7 @@ def main():
     if args.schedule == "stream":
         kernel = "stream_kernel"
     else:
-        kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024) else "sweep_kernel"
+        kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024 and args.schedule != "sliced") else "sweep_kernel"
     one_launch = kernel != "pipe_sweep_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,

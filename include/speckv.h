@@ -98,7 +98,8 @@ enum {
      * behind the first mismatch, so such a row changes no output.  Results are the same either way. */
     SPECKV_READ_ALL_TARGET_ROWS = 1,
     /* Scheduling hints (results are the same either way): take the stream kernel (persistent CTAs,
-     * position-major order) or the sliced sweep whatever the batch size.  At most one of the two.     */
+     * position-major order) or the sliced sweep whatever the batch size and the logit type (fp32
+     * batches of a few hundred rows otherwise take the bulk-copy ring sweep).  At most one of the two. */
     SPECKV_SCHEDULE_STREAM = 2,
     SPECKV_SCHEDULE_SLICED = 4
 };

@@ -440,7 +440,8 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     // resample kernel that cannot overlap) outweigh its streaming rate: b512_mixed cut to 128 / 256 /
     // 512 rows takes 178 / 317 / 564 us with the ring and 166 / 307 / 581 us without.
 constexpr int kPipeMinB = 384;
-    const bool staged = bt->dtype == SPECKV_F32 && aligned && row_bytes % 16 == 0 && P.B <= kPipeMaxB && P.B >= kPipeMinB;
+    const bool staged = bt->dtype == SPECKV_F32 && aligned && row_bytes % 16 == 0 && P.B <= kPipeMaxB && P.B >= kPipeMinB &&
+                        !(bt->flags & SPECKV_SCHEDULE_SLICED);
     // completion flags per batch row and the logits at the draft tokens: only the register-staged sweep
     // overlaps the resample work with its own tail; after the ring sweep the resample kernel starts when
     // everything is done and a flag would only cost it a round trip
