@@ -403,6 +403,8 @@ def test_ring_sweep_with_padded_rows_and_ragged_ends_fp32():
     flat[1:] = s["target"].flatten()
     s3 = dict(s); s3["target"] = flat[1:].view_as(s["target"])
     compare_step(speckv.speckv_step(gpu_batch(s3), s["comp"], gm), ref)
+    # the same aligned batch through the sliced sweep, asked for by flag
+    compare_step(speckv.speckv_step(gpu_batch(s, flags=binding.SCHEDULE_SLICED), s["comp"], gm), ref)
 
 
 @pytest.mark.parametrize("name,B,V", [("b256", 16, 128256), ("b512_mixed", 16, 151936), ("b512_mixed", 400, 8000)])
