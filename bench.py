@@ -238,7 +238,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-early-exit", action="store_true",
                     help="read every target row (SPECKV_READ_ALL_TARGET_ROWS): the all-positions reference for GB/s")
-    ap.add_argument("--schedule", default="auto", choices=["auto", "stream", "sliced"], help="kernel choice hint passed to the library")
+    ap.add_argument("--schedule", default="auto", choices=["auto", "sliced"], help="kernel choice hint passed to the library")
     ap.add_argument("--min-seconds", type=float, default=0.5, help="the timed blocks are repeated until this much time has passed")
     ap.add_argument("--dry-run", action="store_true", help="exercise the launcher and the rank plumbing on CPU (gloo), no kernels")
     args = ap.parse_args()
@@ -277,7 +277,7 @@ def main():
 
     from paper_2605_02888_b200 import binding as _b
     flags = (_b.READ_ALL_TARGET_ROWS if args.no_early_exit else 0) | \
-            {"auto": 0, "stream": _b.SCHEDULE_STREAM, "sliced": _b.SCHEDULE_SLICED}[args.schedule]
+            {"auto": 0, "sliced": _b.SCHEDULE_SLICED}[args.schedule]
 
     def gpu_batch(s):
         return speckv.Batch(draft_logits=s["draft"], target_logits=s["target"], draft_tokens=s["draft_tokens"],
@@ -368,10 +368,7 @@ def main():
     # the library picks by logit type and batch: fp32, 384..1024 rows -> ring sweep, then a resample kernel (two launches per step);
     # bf16 -> register-staged sweep whose grid also carries the resample CTAs (one launch per step, so
     # its duration is that of the whole pass over the batch, second read of the stop positions included)
-    if args.schedule == "stream":
-        kernel = "stream_kernel"
-    else:
-        kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024 and args.schedule != "sliced") else "sweep_kernel"
+    kernel = "pipe_sweep_kernel" if (w.dtype == "fp32" and 384 <= wr.B <= 1024 and args.schedule != "sliced") else "sweep_kernel"
     one_launch = kernel != "pipe_sweep_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": ncu_traffic_bytes(kernel, w.name) if not args.rows else None,

@@ -97,10 +97,9 @@ enum {
      * that is already known to be rejected is left out: Sec. 3.1 discards what the target produced
      * behind the first mismatch, so such a row changes no output.  Results are the same either way. */
     SPECKV_READ_ALL_TARGET_ROWS = 1,
-    /* Scheduling hints (results are the same either way): take the stream kernel (persistent CTAs,
-     * position-major order) or the sliced sweep whatever the batch size and the logit type (fp32
-     * batches of a few hundred rows otherwise take the bulk-copy ring sweep).  At most one of the two. */
-    SPECKV_SCHEDULE_STREAM = 2,
+    /* Scheduling hint (results are the same either way): take the sliced sweep whatever the batch size
+     * and the logit type (fp32 batches of a few hundred rows otherwise take the bulk-copy ring sweep).
+     * The value 2 is not in use: a batch that sets it is rejected with SPECKV_ERR_INVALID_ARG.          */
     SPECKV_SCHEDULE_SLICED = 4
 };
 

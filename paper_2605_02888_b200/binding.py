@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_STATIC_LIMIT 
 F32, BF16 = 0, 1
 ROW_OK, ROW_BAD_GAMMA, ROW_BAD_TOKEN, ROW_NONFINITE, ROW_BAD_TEMPERATURE, ROW_TIMEOUT = 0, 1, 2, 4, 8, 16
 
-READ_ALL_TARGET_ROWS, SCHEDULE_STREAM, SCHEDULE_SLICED = 1, 2, 4   # speckv_batch.flags
+READ_ALL_TARGET_ROWS, SCHEDULE_SLICED = 1, 4   # speckv_batch.flags
 
 STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ("speckv_workspace_size", "speckv_signals", "speckv_signals_static", "speckv_select_gamma", "speckv_verify",
@@ -162,7 +162,7 @@ class Batch:
     temperature_scalar: float = 1.0
     uniforms: Optional[torch.Tensor] = None         # [B, gamma_max+1, 2] fp32
     entropy_in_bits: bool = False
-    flags: int = 0                                  # READ_ALL_TARGET_ROWS | SCHEDULE_STREAM | SCHEDULE_SLICED
+    flags: int = 0                                  # READ_ALL_TARGET_ROWS | SCHEDULE_SLICED
 
     def shape(self):
         B, G, V = self.draft_logits.shape

@@ -10,8 +10,7 @@ _CSRC = os.path.join(_PKG, "csrc")
 _INC = os.path.join(os.path.dirname(_PKG), "include")
 LIB_PATH = os.path.join(_CSRC, "libspeckv.so")
 _SOURCES = ["speckv.cu"]
-_DEPS = ["speckv.cu", "speckv_kernels.cuh", "speckv_pipeline.cuh", "speckv_shard.cuh", "speckv_sample.cuh",
-         "speckv_stream.cuh"]
+_DEPS = ["speckv.cu", "speckv_kernels.cuh", "speckv_pipeline.cuh", "speckv_shard.cuh", "speckv_sample.cuh"]
 
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared"]

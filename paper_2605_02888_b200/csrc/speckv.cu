@@ -16,7 +16,6 @@
 #include "speckv_pipeline.cuh"
 #include "speckv_shard.cuh"
 #include "speckv_sample.cuh"
-#include "speckv_stream.cuh"
 
 namespace {
 
@@ -24,9 +23,7 @@ using namespace speckv;
 
 constexpr int kSliceBytes = 262144;  // bytes of one logit row that one sweep CTA streams
 constexpr size_t kAlign = 256;
-// upper bound of a verification step's logit bytes from which the stream kernel is taken
-constexpr long long kStreamMinBytes = 128ll << 20;
-constexpr bool kStreamByDefault = false;  // until it outruns the sliced sweep on the large batches
+
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct Plan {
@@ -113,56 +110,8 @@ Plan make_plan(const speckv_batch* bt) {
     return p;
 }
 
-// Workspace of the stream kernel (speckv_stream.cuh).  Depends on the batch shape only.
-struct StreamPlan {
-    bool fits;        // the shape is one the stream kernel takes
-    int n_slice, slice_elems, rs_shares, nchunk;
-    size_t off_ctrl, off_state, off_ptick, off_tick2, off_rsq, zero_bytes;  // [0, zero_bytes) is cleared per call
-    size_t off_info, off_pos, off_fresh, off_part, off_csum, total;
-};
-
-StreamPlan make_stream_plan(const speckv_batch* bt) {
-    StreamPlan p{};
-    const size_t B = static_cast<size_t>(bt->B), G1 = static_cast<size_t>(bt->gamma_max) + 1;
-    // slices per logit row: none for large batches; small batches are cut so that the SMs have a few
-    // items each; a slice holds at most kSMaxQ warp quanta
-    const long long max_slice = static_cast<long long>(kSMaxQ) * kSQElems;
-    long long ns = (bt->V + max_slice - 1) / max_slice;
-    const long long rows = static_cast<long long>(bt->B) * (2 * bt->gamma_max + 1);
-    const long long want = rows > 0 ? (4 * 148 + rows - 1) / rows : 1;
-    if (want > ns) ns = want;
-    if (ns > kSMaxSlice) ns = kSMaxSlice;
-    long long se = (bt->V + ns - 1) / ns;
-    se = (se + kSQElems - 1) / kSQElems * kSQElems;
-    ns = (bt->V + se - 1) / se;
-    p.n_slice = static_cast<int>(ns);
-    p.slice_elems = static_cast<int>(se);
-    p.nchunk = (bt->V + kChunk - 1) / kChunk;
-    p.rs_shares = (p.nchunk + kSRsShare - 1) / kSRsShare;
-    p.fits = bt->B <= kSMaxB && se <= max_slice && ns <= kSMaxSlice && bt->V <= (1 << 28) &&
-             static_cast<long long>(bt->B) * G1 * 2 * ns <= 0x7fffffffLL / 4;
-    size_t off = 0;
-    p.off_ctrl = off; off = align_up(off + sizeof(SCtrl));
-    p.off_state = off; off = align_up(off + B * sizeof(unsigned long long));
-    p.off_ptick = off; off = align_up(off + B * G1 * sizeof(int));
-    p.off_tick2 = off; off = align_up(off + B * sizeof(int));
-    p.off_rsq = off; off = align_up(off + B * sizeof(int));
-    p.zero_bytes = off;
-    p.off_info = off; off = align_up(off + B * sizeof(RowInfo));
-    p.off_pos = off; off = align_up(off + B * G1 * sizeof(PosRec));
-    p.off_fresh = off; off = align_up(off + B * sizeof(int));
-    p.off_part = off; off = align_up(off + B * G1 * 2 * static_cast<size_t>(ns) * sizeof(float4));
-    p.off_csum = off; off = align_up(off + B * static_cast<size_t>(p.nchunk) * sizeof(float));
-    p.total = off;
-    return p;
-}
-
-// what the caller must provide: enough for whichever kernel the call takes
-size_t workspace_total(const speckv_batch* bt) {
-    const Plan a = make_plan(bt);
-    const StreamPlan b = make_stream_plan(bt);
-    return (b.fits && b.total > a.total) ? b.total : a.total;
-}
+// what the caller must provide
+size_t workspace_total(const speckv_batch* bt) { return make_plan(bt).total; }
 
 // polls a waiting CTA spends before it gives a row up (SPECKV_ROW_TIMEOUT); lowered by tests only
 std::atomic<int> g_wait_limit{1 << 20};
@@ -183,8 +132,7 @@ speckv_status check_batch(const speckv_batch* bt, bool need_target) {
         if (!stride_ok(bt->target_stride_b) || !stride_ok(bt->target_stride_pos)) return SPECKV_ERR_INVALID_ARG;
     }
     if (!(bt->temperature) && !(bt->temperature_scalar >= 0.f)) return SPECKV_ERR_INVALID_ARG;
-    if (bt->flags & ~(SPECKV_READ_ALL_TARGET_ROWS | SPECKV_SCHEDULE_STREAM | SPECKV_SCHEDULE_SLICED)) return SPECKV_ERR_INVALID_ARG;
-    if ((bt->flags & SPECKV_SCHEDULE_STREAM) && (bt->flags & SPECKV_SCHEDULE_SLICED)) return SPECKV_ERR_INVALID_ARG;
+    if (bt->flags & ~(SPECKV_READ_ALL_TARGET_ROWS | SPECKV_SCHEDULE_SLICED)) return SPECKV_ERR_INVALID_ARG;
     return SPECKV_OK;
 }
 
@@ -305,30 +253,6 @@ cudaError_t launch_all(KParams P, cudaStream_t st, const Events& ev, bool staged
     return e;
 }
 
-// The stream kernel: one persistent CTA per SM (speckv_stream.cuh).
-template <typename T>
-cudaError_t launch_stream(const KParams& P, const SParams& S, cudaStream_t st, const Events& ev) {
-    static std::atomic<bool> configured[64];
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    const bool slot = dev >= 0 && dev < 64;
-    if (!slot || !configured[dev].load(std::memory_order_acquire)) {
-        e = cudaFuncSetAttribute(stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSDynBytes);
-        if (e != cudaSuccess) return e;
-        if (slot) configured[dev].store(true, std::memory_order_release);
-    }
-    int sms = 0;
-    e = sm_count(&sms);
-    if (e != cudaSuccess) return e;
-    if (ev.before_sweep) cudaEventRecord(ev.before_sweep, st);
-    stream_kernel<T><<<sms, kSThreads, kSDynBytes, st>>>(P, S);
-    e = cudaGetLastError();
-    if (ev.after_sweep) cudaEventRecord(ev.after_sweep, st);
-    if (ev.after_resample) cudaEventRecord(ev.after_resample, st);
-    return e;
-}
-
 // Shared driver of signals / verify / step.
 speckv_status run(const speckv_batch* bt, int mode, const float* comp, const speckv_mlp* mlp, float* H,
                   float* C, float* feat, float* scores, int32_t* gamma_next, int32_t* n_accepted,
@@ -395,37 +319,6 @@ speckv_status run(const speckv_batch* bt, int mode, const float* comp, const spe
     bool aligned = rows_aligned(bt->draft_logits, bt->draft_stride_b, bt->draft_stride_pos, es);
     if (verify) aligned = aligned && rows_aligned(bt->target_logits, bt->target_stride_b, bt->target_stride_pos, es);
     const long long row_bytes = static_cast<long long>(P.V) * es;
-
-    // Verification of batches with enough logit rows to keep every SM streaming goes to the stream kernel
-    // (position-major order, early exit behind a rejection, draws from L2); smaller ones, signals alone
-    // and rows that are not whole 16-byte granules take the sliced sweep below.
-    {
-        const StreamPlan sp = make_stream_plan(bt);
-        const long long upper_bytes = static_cast<long long>(P.B) * pl.J_full * row_bytes;
-        const bool big = upper_bytes >= kStreamMinBytes;
-        const bool want = (bt->flags & SPECKV_SCHEDULE_STREAM) ||
-                          (kStreamByDefault && !(bt->flags & SPECKV_SCHEDULE_SLICED) && big && bt->dtype == SPECKV_BF16);
-        if (verify && want && sp.fits && aligned && row_bytes % 16 == 0) {
-            if (cudaMemsetAsync(ws, 0, sp.zero_bytes, cs) != cudaSuccess) return SPECKV_ERR_CUDA;
-            SParams S{};
-            S.n_slice = sp.n_slice; S.slice_elems = sp.slice_elems; S.rs_shares = sp.rs_shares;
-            S.read_all = (bt->flags & SPECKV_READ_ALL_TARGET_ROWS) ? 1 : 0;
-            S.ctrl = reinterpret_cast<SCtrl*>(w + sp.off_ctrl);
-            S.state = reinterpret_cast<unsigned long long*>(w + sp.off_state);
-            S.ptick = reinterpret_cast<int*>(w + sp.off_ptick);
-            S.rsq = reinterpret_cast<int*>(w + sp.off_rsq);
-            S.pos = reinterpret_cast<PosRec*>(w + sp.off_pos);
-            S.fresh = reinterpret_cast<int*>(w + sp.off_fresh);
-            S.poll_limit = P.wait_limit;
-            P.tick2 = reinterpret_cast<int*>(w + sp.off_tick2);
-            P.info = reinterpret_cast<RowInfo*>(w + sp.off_info);
-            P.part = reinterpret_cast<float4*>(w + sp.off_part);
-            P.csum = reinterpret_cast<float*>(w + sp.off_csum);
-            const cudaError_t e = bt->dtype == SPECKV_BF16 ? launch_stream<__nv_bfloat16>(P, S, cs, ev)
-                                                          : launch_stream<float>(P, S, cs, ev);
-            return e == cudaSuccess ? SPECKV_OK : SPECKV_ERR_CUDA;
-        }
-    }
 
     if (cudaMemsetAsync(P.tick1, 0, (6 * static_cast<size_t>(P.B) + 4) * sizeof(int), cs) != cudaSuccess)
         return SPECKV_ERR_CUDA;

@@ -2,7 +2,7 @@
 logit load and every workspace access of every kernel is compared with the extents of the call's buffers
 and an access outside them is skipped and counted, never performed.  The shapes most likely to expose an
 index mistake go through it here - vocabularies that are not a multiple of anything, ragged gamma, padded
-and misaligned rows, broadcast rows (stride 0), the ring sweep's ragged stages, the stream kernel, the
+and misaligned rows, broadcast rows (stride 0), the ring sweep's ragged stages, every target row read, the
 sharded step, draft sampling - and the count must stay at zero with results that match the oracle.  A
 self-test has the checker look at two addresses that no call registered (they are compared, not
 dereferenced) to show that it would have counted them."""
@@ -65,8 +65,7 @@ def test_no_access_leaves_its_buffers(debug_library):
             w = synth.Workload("d", B=B, gamma_max=G, V=V, dtype=dtype, gamma_mode="ragged", temperature_mode="mixed",
                                sigma_d=synth.SIGMA_LEVELS, frac_onehot=0.2, seed=V)
             _check(w)
-            if V % 8 == 0:
-                _check(w, flags=binding.SCHEDULE_STREAM)
+            _check(w, flags=binding.READ_ALL_TARGET_ROWS)
     assert _violations(L)[0] == 0, _violations(L)
     # a single batch row cut into many slices: more partials per logit row than the epilogue fetches ahead,
     # and nothing behind the row's partials but the end of the array
@@ -75,11 +74,13 @@ def test_no_access_leaves_its_buffers(debug_library):
                            sigma_d=(0.6,), seed=50)
         _check(w)
     assert _violations(L)[0] == 0, _violations(L)
-    # the stream kernel with several slices per row, and with more than 32 quanta per item
-    for dtype, V in (("bf16", 300000), ("fp32", 40000)):
-        w = synth.Workload("d", B=6, gamma_max=3, V=V, dtype=dtype, gamma_mode="ragged", temperature=0.8,
+    # long rows in several slices, and enough batch rows of one slice each for the later generations of the grid
+    # to find stop positions published (target rows left unread)
+    for dtype, V, B in (("bf16", 300000, 6), ("fp32", 40000, 6), ("bf16", 32000, 300)):
+        w = synth.Workload("d", B=B, gamma_max=3, V=V, dtype=dtype, gamma_mode="ragged", temperature=0.8,
                            sigma_d=(0.6,), seed=3)
-        _check(w, flags=binding.SCHEDULE_STREAM)
+        _check(w)
+        _check(w, flags=binding.SCHEDULE_SLICED | binding.READ_ALL_TARGET_ROWS)
     assert _violations(L)[0] == 0, _violations(L)
     # the ring sweep (fp32, 384 rows and more) with rows that are not whole stages
     w = synth.Workload("d", B=400, gamma_max=2, V=4100, dtype="fp32", gamma_mode="ragged", temperature=0.9,

@@ -471,11 +471,11 @@ def test_target_rows_behind_a_rejection_are_skipped_without_changing_anything(B,
 
 
 @pytest.mark.parametrize("name,B,V,flags", [("b256", 64, 32000, 0), ("b512_mixed", 400, 8000, 0), ("b512_mixed", 32, 8000, 0),
-                                            ("b256", 64, 32000, 2)])
+                                            ("b512_mixed", 400, 8000, 4)])
 def test_step_can_be_captured_in_a_cuda_graph(name, B, V, flags):
     # the library only enqueues work on the caller's stream (no allocation, no synchronisation), so a step
     # can be recorded once and replayed: single-launch path, ring sweep + dependent resample kernel, fp32 fallback,
-    # and the stream kernel (flags = 2, SPECKV_SCHEDULE_STREAM)
+    # and the sliced sweep asked for by flag for a batch that would take the ring (flags = 4, SPECKV_SCHEDULE_SLICED)
     w = synth.scaled(synth.WORKLOADS[name], B=B, V=V)
     s = synth.make_step(w, 0, DEV)
     gm, _ = mlp_pair(synth.make_mlp(w, DEV))

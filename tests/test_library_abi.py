@@ -62,6 +62,9 @@ def test_workspace_size_and_argument_checks_without_a_gpu():
     assert call(_cb(), 0x101, 1 << 30) == binding.ERR_INVALID_ARG
     assert call(_cb(), 0x100, 16) == binding.ERR_WORKSPACE
     assert call(_cb(B=-1), 0x100, 1 << 30) == binding.ERR_INVALID_ARG
+    # flags: the value 2 (no kernel behind it any more) and unknown bits are refused before anything is launched
+    assert call(_cb(flags=2), 0x100, 1 << 30) == binding.ERR_INVALID_ARG
+    assert call(_cb(flags=8), 0x100, 1 << 30) == binding.ERR_INVALID_ARG
     assert call(_cb(B=0), None, 0) == binding.OK          # empty batch: nothing to do
     # verify needs target, tokens and uniforms
     assert L.speckv_verify(C.byref(_cb()), 0x100, 0x100, None, 0x100, 1 << 30, None) == binding.ERR_INVALID_ARG
