@@ -102,8 +102,11 @@ __device__ __forceinline__ bool mbar_test(unsigned long long* bar, uint32_t pari
     return ok != 0;
 }
 // Bounded wait for the phase with the given parity; false when the limit ran out or the CTA's
-// error flag is up.
+// error flag is up.  The bound is a time (about two seconds on the GPU's nanosecond clock), not a number of
+// tries: one try may come back at once or only when the hardware's own limit for a try is up.
+constexpr unsigned long long kWaitNs = 2000000000ull;
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* error) {
+    unsigned long long t0 = 0;
     for (int it = 0; it < kWaitLimit; ++it) {
         uint32_t ok;
         asm volatile(
@@ -112,7 +115,11 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
             : "r"(smem_u32(bar)), "r"(parity)
             : "memory");
         if (ok) return true;
-        if ((it & 1023) == 1023 && *error) return false;
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        else if (now - t0 > kWaitNs) break;
+        if ((it & 63) == 63 && *error) return false;
     }
     *error = 1;
     return false;
