@@ -205,7 +205,7 @@ cudaError_t launch_pipe(const KParams& P, cudaStream_t st) {
 }
 
 // After the register-staged sweep the fresh tokens are drawn by extra CTAs of the same launch; the rows swept last have their fresh tokens drawn by more, shorter CTAs (see resample_body)
-constexpr int kRsTailRows = 16;
+constexpr int kRsTailRows = 32;  // b256, same box, builds in turn: 16 rows 158.7 us, 32 rows 156.6 us, 64 rows 156.7 us, 128 rows 157.2 us
 constexpr int kRsTailMult = 2;
 constexpr int kRsSmallCtas = 1184;  // resample CTAs wanted in flight for a small batch (two per CTA slot)
 
